@@ -1,0 +1,245 @@
+/*
+ * samdraft.h — C ABI of libsamdraft: batched suffix-automaton draft retrieval on one GPU.
+ *
+ * The library implements the draft-retrieval path of SAM-Decoding (arXiv 2411.10666) for a batch
+ * of decoding sequences:
+ *   - a STATIC suffix automaton over a token corpus, built offline on the host (Build-SAM,
+ *     Algorithm 3) and stored on the device;
+ *   - one DYNAMIC suffix automaton per sequence, extended on the device with every accepted
+ *     token (Expand, Algorithm 3) after the sequence's match state has been advanced on the
+ *     automaton as it was (Transfer, Algorithm 1; order of Section 3.3);
+ *   - the draft d = T[p+1 : p+n] read after the first end position p (min_endpos, Section 3.1)
+ *     of the matched state, from the static text iff l1 > l2 + l_bias (Section 3.2).
+ *
+ * Conventions
+ *   - Every function returns 0 on success or a negative sam_err_t; none aborts or throws.
+ *   - "host" / "device" in a parameter comment says where the pointed-to memory must live.
+ *     Device pointers must belong to the device the object was created on.
+ *   - Tokens are int32 in [0, vocab).  Positions reported by the paper's algorithms are 1-based;
+ *     nothing 1-based crosses this interface (only tokens, lengths and state ids do).
+ *   - State ids are creation-order ids of Algorithm 3: root 0, each new state before its clone.
+ *   - All device work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL
+ *     is the legacy default stream) and is asynchronous unless stated otherwise.
+ *   - Objects are not thread-safe; calls on one sam_batch_t must be externally ordered.
+ */
+#ifndef SAMDRAFT_H
+#define SAMDRAFT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SAM_OK = 0,
+    SAM_ERR_ARG = -1,        /* null pointer, size out of range, inconsistent options        */
+    SAM_ERR_CUDA = -2,       /* a CUDA runtime call failed (sam_last_cuda_error has its code)  */
+    SAM_ERR_NOMEM = -3,      /* host or device allocation failed                              */
+    SAM_ERR_WORKSPACE = -4,  /* caller's workspace too small or misaligned                    */
+    SAM_ERR_IO = -5,         /* file could not be read / written                              */
+    SAM_ERR_FORMAT = -6,     /* file is not a static-automaton image, or its checksum is bad  */
+    SAM_ERR_LIMIT = -7,      /* corpus or option exceeds what the layout can index            */
+    SAM_ERR_NO_DEVICE = -8   /* no usable CUDA device                                         */
+} sam_err_t;
+
+/* Per-sequence status written by sam_step (status_dev).  Non-zero is sticky until reset. */
+enum {
+    SAM_SEQ_OK = 0,
+    SAM_SEQ_CAPACITY = 1,    /* seq_len + count > max_seq_len, or the slab pool ran dry       */
+    SAM_SEQ_WALK_LIMIT = 2,  /* a bounded probe / link walk hit its limit (corrupt state)     */
+    SAM_SEQ_BAD_TOKEN = 3,   /* a token outside [0, vocab)                                    */
+    SAM_SEQ_BAD_COUNT = 4    /* count < 0 or count > stride                                   */
+};
+
+/* source_dev values */
+enum { SAM_SRC_NONE = 0, SAM_SRC_STATIC = 1, SAM_SRC_DYNAMIC = 2 };
+
+typedef struct sam_static sam_static_t;   /* device-resident static automaton, owned by the library */
+typedef struct sam_batch sam_batch_t;     /* batch of sequences; its device memory is the caller's  */
+
+typedef struct {
+    double hash_load;        /* target load of the overflow-edge hash table, (0, 0.9]; 0 = 0.5 */
+    int32_t keep_host_copy;  /* reserved, must be 0                                            */
+} sam_build_opts_t;
+
+typedef struct {
+    int64_t n_tokens;        /* corpus length                                                  */
+    int64_t n_states;        /* states of the automaton (<= 2 n_tokens - 1)                    */
+    int64_t n_transitions;   /* transitions (<= 3 n_tokens - 4)                                */
+    int64_t n_hash_edges;    /* transitions stored in the overflow hash table                  */
+    int64_t hash_buckets;    /* 128-byte buckets of that table                                 */
+    int32_t hash_max_probe;  /* longest bucket probe sequence any stored edge needs            */
+    int32_t vocab;
+    size_t device_bytes;     /* device memory held                                             */
+    double build_seconds;    /* host construction time (0 for a loaded image)                  */
+} sam_static_info_t;
+
+typedef struct {
+    int32_t batch;            /* number of sequence slots B, >= 1                              */
+    int32_t max_seq_len;      /* most tokens (prompt + accepted) a slot may hold, >= 1         */
+    int32_t max_draft_len;    /* largest L any sam_step will ask for, 1..128                   */
+    int32_t l_bias;           /* static wins iff l1 > l2 + l_bias (Section 3.2); >= 0          */
+    int32_t min_match;        /* a chosen match shorter than max(1, min_match) gives no draft  */
+    int32_t vocab;            /* token range when there is no static automaton, else ignored   */
+    int32_t max_host_stride;  /* largest stride sam_step_host accepts; 0 = 32                  */
+    int32_t slab_bytes;       /* slab size, a power of two >= 4 KiB; 0 = max(16 KiB, pow2 >= 8*max_seq_len) */
+    int64_t pool_slabs;       /* slabs in the shared pool; 0 = batch * (ceil(160 * max_seq_len / slab_bytes) + 2) */
+} sam_batch_opts_t;
+
+/* ---- static automaton -------------------------------------------------------------------- */
+
+/* Build-SAM (Algorithm 3) over corpus_host[0, n_tokens) on the host, then store the result on
+ * `device`: one 32-byte record per state (length, link, min_endpos and up to two transitions
+ * inline), a dense row for the root, a bucketed (state, token) hash table for the remaining
+ * transitions, and the corpus itself for draft reads.  Synchronous; this is the offline step.
+ * corpus_host: host, n_tokens int32, each in [0, vocab); not retained.  opts may be NULL.
+ * *out is owned by the library; release it with sam_static_destroy.
+ * Errors: ARG (null, n_tokens < 1, vocab < 1, token out of range), LIMIT (n_tokens > 2^30),
+ * NOMEM, CUDA. */
+int sam_build_static(const int32_t* corpus_host, int64_t n_tokens, int32_t vocab, int device,
+                     const sam_build_opts_t* opts, sam_static_t** out);
+
+/* Write / read the device image of a built automaton so large corpora are indexed once.
+ * The file holds a header (magic, version, sizes, FNV-1a checksum of the payload) and the raw
+ * sections.  Both calls are synchronous.  Errors: ARG, IO, FORMAT, NOMEM, CUDA. */
+int sam_static_save(const sam_static_t* st, const char* path);
+int sam_static_load(const char* path, int device, sam_static_t** out);
+
+int sam_static_info(const sam_static_t* st, sam_static_info_t* out);
+
+/* Copy one state's record back to the host (synchronous; for inspection and tests).
+ * next_tokens / next_targets receive up to max_edges of the state's transitions in no particular
+ * order; *n_edges gets the state's out-degree (which may exceed max_edges).
+ * For the root only the out-degree is reported through this call's edge arrays when max_edges
+ * is smaller than it.  Errors: ARG (state out of range), CUDA. */
+int sam_static_state(const sam_static_t* st, int64_t state, int32_t* length, int32_t* link,
+                     int32_t* min_endpos, int32_t* n_edges,
+                     int32_t* next_tokens, int32_t* next_targets, int32_t max_edges);
+
+/* Copy length, link (root: -1), min_endpos and out-degree of the first max_states states to the
+ * host (synchronous; inspection and tests).  Errors: ARG, NOMEM, CUDA. */
+int sam_static_tables(const sam_static_t* st, int32_t* length, int32_t* link, int32_t* min_endpos,
+                      int32_t* deg, int64_t max_states);
+
+/* HOST ONLY, no device needed: run the same construction as sam_build_static and decode the image
+ * it would upload (inline transitions, root row, hash buckets) back into flat tables; also checks
+ * the image's internal consistency (hash reachability, has-hashed-transitions bits) and returns
+ * FORMAT if that fails.  Arrays may be NULL to get the counts only.  For tests and inspection.
+ * Errors: ARG, LIMIT, NOMEM, FORMAT. */
+int sam_build_static_tables(const int32_t* corpus_host, int64_t n_tokens, int32_t vocab,
+                            int64_t* n_states, int64_t* n_transitions, int32_t* hash_max_probe,
+                            int32_t* length, int32_t* link, int32_t* min_endpos, int32_t* deg,
+                            int64_t max_states,
+                            int32_t* edge_src, int32_t* edge_tok, int32_t* edge_tgt, int64_t max_edges);
+
+void sam_static_destroy(sam_static_t* st);
+
+/* ---- batch of sequences ------------------------------------------------------------------- */
+
+/* Bytes of device workspace a batch with these options needs (256-byte aligned base).
+ * Errors: ARG. */
+int sam_batch_workspace_bytes(const sam_batch_opts_t* opts, size_t* out);
+
+/* Lay a batch out in workspace_dev (device memory the CALLER owns and must keep alive and
+ * untouched until sam_batch_destroy) and initialise every slot to the empty sequence: empty
+ * dynamic automaton, both matchers at the root.  st may be NULL (no static source: l1 = 0).
+ * The per-sequence dynamic automata take their state records and edge blocks from a pool of
+ * slabs shared by all slots, handed out on demand.  Initialisation kernels run on `stream`.
+ * Errors: ARG, WORKSPACE (too small / base not 256-byte aligned), NOMEM, CUDA. */
+int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* opts,
+                     void* workspace_dev, size_t workspace_bytes, void* stream, sam_batch_t** out);
+
+/* Return slots to the empty sequence and their slabs to the pool (continuous batching).
+ * slots_host: host, n slot indices; NULL with n < 0 resets every slot.  Errors: ARG, CUDA. */
+int sam_batch_reset(sam_batch_t* b, const int32_t* slots_host, int32_t n, void* stream);
+
+/* One decoding step for all B slots (Sections 3.2, 3.3).  For slot i with m = counts[i]:
+ * each of new_tokens[i, 0..m) is fed, in order, to Transfer on the static automaton, and to
+ * Transfer-then-Expand on the slot's dynamic automaton; then the source is chosen and up to L
+ * draft tokens are read.  m = 0 changes nothing and re-emits the draft of the current state; the
+ * prompt is fed the same way (m = prompt length).
+ *
+ *   new_tokens_dev  device, int32 [B, stride]          counts_dev  device, int32 [B]
+ *   L               1..max_draft_len
+ *   draft_tokens_dev device, int32 [B, L]   drafted tokens, -1 from draft_len on
+ *   draft_len_dev    device, int32 [B]      min(L, tokens that follow the first end position)
+ *   match_len_dev    device, int32 [B, 2]   (l1 static, l2 dynamic)
+ *   source_dev       device, int32 [B]      SAM_SRC_*
+ *   state_dev        device, int32 [B, 2]   (static state, dynamic state); may be NULL
+ *   status_dev       device, int32 [B]      SAM_SEQ_*; a failed slot reports zeros and -1 drafts
+ *
+ * Host-visible argument errors (null, L out of range, stride < 1) return ARG synchronously and
+ * launch nothing; data-dependent problems are reported per slot in status_dev and freeze the
+ * slot until it is reset.  A slot is validated (count, capacity, token range) before any of its
+ * state changes. */
+int sam_step(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
+             const int32_t* counts_dev, int32_t L,
+             int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,
+             int32_t* source_dev, int32_t* state_dev, int32_t* status_dev, void* stream);
+
+/* Replay n_steps consecutive steps from device arrays without returning to the caller in
+ * between: new_tokens_dev [n_steps, B, stride], counts_dev [n_steps, B].  If out_per_step is
+ * non-zero every output array has a leading n_steps dimension and keeps each step's results,
+ * otherwise the arrays are those of sam_step and hold the last step's.  One kernel launch per
+ * step, same kernel as sam_step. */
+int sam_run_steps(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
+                  const int32_t* counts_dev, int32_t n_steps, int32_t L, int32_t out_per_step,
+                  int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,
+                  int32_t* source_dev, int32_t* state_dev, int32_t* status_dev, void* stream);
+
+/* sam_step with HOST arrays: copies new_tokens and counts to the device, runs the step, copies
+ * every output back and waits for the stream — the end-to-end call a serving loop that keeps its
+ * tokens on the host would make.  stride <= max_host_stride.  Pinned host buffers make the
+ * copies asynchronous with respect to other streams; pageable ones work too.  state_host may be
+ * NULL.  Synchronous.  Errors: as sam_step, plus CUDA. */
+int sam_step_host(sam_batch_t* b, const int32_t* new_tokens_host, int32_t stride,
+                  const int32_t* counts_host, int32_t L,
+                  int32_t* draft_tokens_host, int32_t* draft_len_host, int32_t* match_len_host,
+                  int32_t* source_host, int32_t* state_host, int32_t* status_host, void* stream);
+
+/* Copy slot's dynamic automaton to the host (synchronous; inspection and tests).
+ * length/link/min_endpos/deg: host, max_states int32 each; edge_src/edge_tok/edge_tgt: host,
+ * max_edges int32 each.  *n_states / *n_edges receive the true counts; arrays are filled up to
+ * their capacity.  Errors: ARG, NOMEM, CUDA. */
+int sam_batch_dump(sam_batch_t* b, int32_t slot, int32_t* n_tokens, int32_t* n_states,
+                   int32_t* n_edges, int32_t* length, int32_t* link, int32_t* min_endpos,
+                   int32_t* deg, int32_t max_states,
+                   int32_t* edge_src, int32_t* edge_tok, int32_t* edge_tgt, int32_t max_edges,
+                   void* stream);
+
+/* Pool occupancy: slabs in the pool, slabs currently free.  Synchronous. */
+int sam_batch_pool_info(sam_batch_t* b, int64_t* total_slabs, int64_t* free_slabs, void* stream);
+
+/* Forget the batch.  The workspace is the caller's and is not freed. */
+void sam_batch_destroy(sam_batch_t* b);
+
+/* ---- memory-system probes (the denominators of the random-access roofline) ---------------- */
+
+/* Independent uniformly random aligned reads of `granule` bytes (32, 64 or 128) over
+ * buf_dev[0, footprint_bytes): every SM full of warps, several loads in flight per thread.
+ * Runs `iters` timed launches after one warm-up; *gbps gets bytes read / best time, *mreq_s the
+ * matching requests per microsecond.  buf_dev: device, footprint_bytes, caller-owned (contents
+ * irrelevant).  Synchronous.  Errors: ARG, CUDA. */
+int sam_probe_random_read(void* buf_dev, size_t footprint_bytes, int32_t granule, int32_t iters,
+                          void* stream, double* gbps, double* mreq_s);
+
+/* Dependent-load latency: `chains` single-thread chains (one per block, 1..65536) each chase a
+ * random cyclic permutation of the 128-byte lines of buf_dev[0, footprint_bytes) for `hops` hops,
+ * starting at evenly spaced points of the cycle; *ns_per_hop gets the time per hop of one chain
+ * (so chains / ns_per_hop is the rate of dependent reads at that concurrency).  The permutation is
+ * written into buf_dev by this call.  Synchronous.  Errors: ARG, NOMEM, CUDA. */
+int sam_probe_chase(void* buf_dev, size_t footprint_bytes, int64_t hops, int32_t chains,
+                    void* stream, double* ns_per_hop);
+
+/* ---- diagnostics --------------------------------------------------------------------------- */
+
+const char* sam_strerror(int err);
+int sam_last_cuda_error(void);          /* cudaError_t of the last failed runtime call, else 0 */
+const char* sam_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAMDRAFT_H */

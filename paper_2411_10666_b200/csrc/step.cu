@@ -1,0 +1,535 @@
+// The hot kernel: one decoding step of SAM-Decoding's draft retrieval for a batch of sequences.
+//
+// One block of two warps per sequence slot.  Warp 0 advances the slot's match state through the
+// STATIC automaton (Transfer, Algorithm 1) for each accepted token; warp 1 extends the slot's own
+// DYNAMIC automaton (Expand, Algorithm 3) with the same tokens and keeps its match state, which
+// after each Expand is link[last] with length len[link[last]] (the state Transfer would reach on
+// the automaton as it was before the token, Section 3.3, made canonical).  Both warps then read
+// the first end position of their state, fetch their candidate draft speculatively, and the
+// source rule l1 > l2 + l_bias (Section 3.2) picks which one is written out.
+//
+// Each warp runs one dependent chain of memory reads, so the work is latency-bound: every value
+// is warp-uniform (all lanes read the same 32-byte record, one request), and the lanes are used
+// side by side only where a structure is wide — a 128-byte hash bucket, a 256-byte root-table
+// bucket, an edge block, the draft read.  Independent reads are issued together (record + hash
+// bucket, root-row entries for all tokens of the step up front).
+#include "common.h"
+
+namespace {
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+constexpr int MAX_DRAFT_REGS = 4;     // 4 x 32 lanes = 128 draft tokens
+
+struct StepArgs {
+    SamStaticView S;
+    SamBatchView W;
+    int32_t has_static;
+    const int32_t* new_tokens; int32_t stride; const int32_t* counts; int32_t L;
+    int32_t* draft_tokens; int32_t* draft_len; int32_t* match_len; int32_t* source;
+    int32_t* state; int32_t* status;
+};
+
+// ------------------------------------------------------------------ draft read
+// d[r] (lane j of round r) = text[e + 32 r + j] for 32 r + j < dl, else -1.  The window is read as
+// aligned 16-byte vectors (nine lanes per 32 tokens) and realigned with shuffles.
+template <bool READONLY>
+__device__ __forceinline__ void gather_draft(const int32_t* text, int64_t e, int dl, int L, int lane,
+                                             int32_t d[MAX_DRAFT_REGS]) {
+    const int off = (int)(e & 3);
+    const int4* v = reinterpret_cast<const int4*>(text + (e - off));
+    const int nvec = (off + dl + 3) >> 2;
+    const int src = (off + lane) >> 2, comp = (off + lane) & 3;
+#pragma unroll
+    for (int r = 0; r < MAX_DRAFT_REGS; r++) {
+        d[r] = -1;
+        if (r * 32 < L) {
+            int4 q = make_int4(0, 0, 0, 0);
+            const int vi = 8 * r + lane;
+            if (lane < 9 && vi < nvec) q = READONLY ? __ldg(v + vi) : v[vi];
+            int x0 = __shfl_sync(FULL, q.x, src), x1 = __shfl_sync(FULL, q.y, src);
+            int x2 = __shfl_sync(FULL, q.z, src), x3 = __shfl_sync(FULL, q.w, src);
+            int val = comp == 0 ? x0 : comp == 1 ? x1 : comp == 2 ? x2 : x3;
+            if (r * 32 + lane < dl) d[r] = val;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ static side
+// Transfer (Algorithm 1) for one token.  (s, sf, l): state, its F bit, match length.
+// root_e is root_row[t], fetched beforehand.
+__device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t& s, uint32_t& sf, int32_t& l,
+                                                uint32_t t, uint32_t root_e, int lane, int& err) {
+    int guard = l + 2;                       // at most l link moves
+    bool len_from_rec = false;
+    for (;;) {
+        if (s == 0) {                        // at the root the match length is 0
+            if (root_e != SAM_NONE) { s = root_e & SAM_IDMASK; sf = root_e >> 31; l = 1; }
+            else l = 0;
+            return;
+        }
+        uint32_t home = sam_hash2(s, t) & S.hash_mask;
+        uint4 ent = make_uint4(SAM_NONE, 0, 0, 0);
+        if (sf) ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+        const uint4 a = __ldg(S.rec + 2 * (size_t)s);
+        const uint4 b = __ldg(S.rec + 2 * (size_t)s + 1);
+        if (len_from_rec) { l = (int32_t)a.x; len_from_rec = false; }
+        uint32_t tgt = SAM_NONE;
+        if (a.w >= 1 && b.x == t) tgt = b.y;
+        else if (a.w >= 2 && b.z == t) tgt = b.w;
+        else if (a.w > 2) {
+            if (!sf) ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+            for (int probe = 1;; probe++) {
+                unsigned hit = __ballot_sync(FULL, ent.x == s && ent.y == t);
+                if (hit) { tgt = __shfl_sync(FULL, ent.z, __ffs(hit) - 1); break; }
+                unsigned empty = __ballot_sync(FULL, ent.x == SAM_NONE);
+                if (empty || probe >= S.hash_max_probe) break;
+                home = (home + 1) & S.hash_mask;
+                ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+            }
+        }
+        if (tgt != SAM_NONE) { s = tgt & SAM_IDMASK; sf = tgt >> 31; l += 1; return; }
+        s = a.y & SAM_IDMASK; sf = a.y >> 31;            // s <- link(s), l <- len(link(s))
+        if (s == 0) l = 0; else len_from_rec = true;
+        if (--guard < 0) { err = SAM_SEQ_WALK_LIMIT; return; }
+    }
+}
+
+// ------------------------------------------------------------------ dynamic side
+struct Dyn {
+    unsigned char* pool;
+    uint2* root;                 // this slot's root table
+    int32_t* text;               // this slot's token text
+    int32_t* pool_hdr; int32_t* free_stack; int32_t* slab_owner;
+    uint32_t* cb;                // this slot's control block
+    uint32_t tab;                // lane i: slab index of state slab i
+    uint32_t n_rec_slabs, n_states, blk_cur, blk_end, root_deg, root_bmask;
+    int slab_shift, rps_shift, seq, lane, err;
+};
+
+struct Look {                    // result of looking a token up in a non-root state
+    uint32_t len, link, deg, b0, b1, b2, b3;
+    uint32_t tgt;                // transition target with its S bit, valid if found
+    uint32_t idx;                // 0 / 1 inline slot, or index in the edge block
+    bool found;
+};
+
+__device__ __forceinline__ uint4* rec_ptr(const Dyn& D, uint32_t s) {
+    uint32_t slab = __shfl_sync(FULL, D.tab, (int)(s >> D.rps_shift));
+    return reinterpret_cast<uint4*>(D.pool + ((size_t)slab << D.slab_shift) +
+                                    ((size_t)(s & ((1u << D.rps_shift) - 1)) << 5));
+}
+__device__ __forceinline__ uint2* blk_ptr(const Dyn& D, uint32_t off) {
+    return reinterpret_cast<uint2*>(D.pool + (size_t)off * 128);
+}
+
+__device__ __forceinline__ int alloc_slab(Dyn& D) {
+    int idx = -1;
+    if (D.lane == 0) {
+        int old = atomicSub(D.pool_hdr, 1);
+        if (old <= 0) atomicAdd(D.pool_hdr, 1);
+        else { idx = D.free_stack[old - 1]; D.slab_owner[idx] = D.seq; }
+    }
+    return __shfl_sync(FULL, idx, 0);
+}
+
+// make sure state id s has a record to live in
+__device__ __forceinline__ void ensure_rec(Dyn& D, uint32_t s) {
+    uint32_t si = s >> D.rps_shift;
+    if (si < D.n_rec_slabs) return;
+    if (si >= SAM_MAX_REC_SLABS) { D.err = SAM_SEQ_CAPACITY; return; }
+    int slab = alloc_slab(D);
+    if (slab < 0) { D.err = SAM_SEQ_CAPACITY; return; }
+    if (D.lane == (int)si) D.tab = (uint32_t)slab;
+    if (D.lane == 0) D.cb[CB_SLABTAB + si] = (uint32_t)slab;
+    D.n_rec_slabs = si + 1;
+}
+
+// edge block of `cap` entries; returns its offset in 128-byte units from the pool base
+__device__ __forceinline__ uint32_t alloc_block(Dyn& D, uint32_t cap) {
+    uint32_t need = cap >> 4, slab_units = 1u << (D.slab_shift - 7);
+    if (need > slab_units) { D.err = SAM_SEQ_CAPACITY; return 0; }
+    if (D.blk_cur + need > D.blk_end) {
+        int slab = alloc_slab(D);
+        if (slab < 0) { D.err = SAM_SEQ_CAPACITY; return 0; }
+        D.blk_cur = (uint32_t)slab << (D.slab_shift - 7);
+        D.blk_end = D.blk_cur + slab_units;
+    }
+    uint32_t off = D.blk_cur;
+    D.blk_cur += need;
+    return off;
+}
+
+__device__ __forceinline__ Look lookup_state(const Dyn& D, uint32_t p, uint32_t t) {
+    const uint4* rp = rec_ptr(D, p);
+    const uint4 a = rp[0], b = rp[1];
+    Look r;
+    r.len = a.x; r.link = a.y; r.deg = a.w; r.b0 = b.x; r.b1 = b.y; r.b2 = b.z; r.b3 = b.w;
+    r.found = false; r.tgt = 0; r.idx = 0;
+    if (a.w <= 2) {
+        if (a.w >= 1 && b.x == t) { r.found = true; r.tgt = b.y; r.idx = 0; }
+        else if (a.w == 2 && b.z == t) { r.found = true; r.tgt = b.w; r.idx = 1; }
+        return r;
+    }
+    const uint2* blk = blk_ptr(D, b.x);
+    for (uint32_t base = 0; base < a.w; base += 32) {
+        uint32_t i = base + D.lane;
+        uint2 e = make_uint2(SAM_NONE, 0);
+        if (i < a.w) e = blk[i];
+        unsigned hit = __ballot_sync(FULL, e.x == t);
+        if (hit) {
+            int src = __ffs(hit) - 1;
+            r.found = true; r.tgt = __shfl_sync(FULL, e.y, src); r.idx = base + src;
+            break;
+        }
+    }
+    return r;
+}
+
+// add the transition (p, t) -> tgt to a non-root state whose record is in lk
+__device__ __forceinline__ void insert_edge(Dyn& D, uint32_t p, const Look& lk, uint32_t t, uint32_t tgt) {
+    uint4* rp = rec_ptr(D, p);
+    uint32_t* rw = reinterpret_cast<uint32_t*>(rp);
+    if (lk.deg < 2) {
+        if (D.lane == 0) {
+            reinterpret_cast<uint2*>(rp)[2 + lk.deg] = make_uint2(t, tgt);
+            rw[3] = lk.deg + 1;
+        }
+    } else if (lk.deg == 2) {
+        uint32_t off = alloc_block(D, SAM_BLOCK_MIN);
+        if (D.err) return;
+        if (D.lane == 0) {
+            uint2* blk = blk_ptr(D, off);
+            blk[0] = make_uint2(lk.b0, lk.b1); blk[1] = make_uint2(lk.b2, lk.b3); blk[2] = make_uint2(t, tgt);
+            rp[1] = make_uint4(off, SAM_BLOCK_MIN, 0, 0);
+            rw[3] = 3;
+        }
+    } else {
+        uint32_t off = lk.b0, cap = lk.b1;
+        if (lk.deg < cap) {
+            if (D.lane == 0) { blk_ptr(D, off)[lk.deg] = make_uint2(t, tgt); rw[3] = lk.deg + 1; }
+        } else {
+            uint32_t noff = alloc_block(D, cap * 2);
+            if (D.err) return;
+            const uint2* ob = blk_ptr(D, off);
+            uint2* nb = blk_ptr(D, noff);
+            for (uint32_t i = D.lane; i < lk.deg; i += 32) nb[i] = ob[i];
+            if (D.lane == 0) {
+                nb[lk.deg] = make_uint2(t, tgt);
+                rp[1] = make_uint4(noff, cap * 2, 0, 0);
+                rw[3] = lk.deg + 1;
+            }
+        }
+    }
+    __syncwarp();
+}
+
+struct RootLook { uint32_t tgt, slot; bool found; };
+
+__device__ __forceinline__ RootLook root_lookup(Dyn& D, uint32_t t) {
+    RootLook r; r.found = false; r.tgt = 0; r.slot = 0;
+    uint32_t bk = sam_hash1(t) & D.root_bmask;
+    for (uint32_t probe = 0; probe <= D.root_bmask; probe++) {
+        uint2 e = D.root[(size_t)bk * SAM_ROOT_BUCKET + D.lane];
+        unsigned hit = __ballot_sync(FULL, e.x == t);
+        if (hit) {
+            int src = __ffs(hit) - 1;
+            r.found = true; r.tgt = __shfl_sync(FULL, e.y, src); r.slot = bk * SAM_ROOT_BUCKET + src;
+            return r;
+        }
+        unsigned empty = __ballot_sync(FULL, e.x == SAM_NONE);
+        if (empty) { r.slot = bk * SAM_ROOT_BUCKET + (__ffs(empty) - 1); return r; }
+        bk = (bk + 1) & D.root_bmask;
+    }
+    D.err = SAM_SEQ_WALK_LIMIT;           // table full: cannot happen with root_cap >= 2 * distinct tokens
+    return r;
+}
+
+// Expand (Algorithm 3) for token t, fused with the dynamic matcher's Transfer.
+// last: state of the whole text; ntok: text length; (s2, l2): match state = link[last], its length.
+__device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, uint32_t& ntok,
+                                           uint32_t& s2, uint32_t& l2) {
+    const uint32_t k = ntok + 1;                       // max_length after this token
+    const uint32_t c = D.n_states;
+    ensure_rec(D, c);
+    if (D.err) return;
+    D.n_states = c + 1;
+
+    uint32_t p;
+    if (last != 0) {
+        // `last` has no transition yet; it gets (t -> c), solid, and its record is complete now
+        uint4* rl = rec_ptr(D, last);
+        if (D.lane == 0) {
+            rl[0] = make_uint4(ntok, s2, ntok, 1);
+            rl[1] = make_uint4(t, c | SAM_FLAG, 0, 0);
+        }
+        __syncwarp();
+        p = s2;                                        // link[last]
+    } else {
+        p = 0;                                         // empty automaton: last is the root
+    }
+
+    // walk the suffix links from p, adding (t -> c) until a state already has t
+    bool found = false, at_root = false;
+    uint32_t qt = 0, plen = 0, root_slot = 0;
+    Look lk;
+    lk.len = lk.link = lk.deg = lk.b0 = lk.b1 = lk.b2 = lk.b3 = lk.tgt = lk.idx = 0; lk.found = false;
+    int guard = (int)k + 2;
+    for (;;) {
+        if (p == 0) {
+            RootLook rl = root_lookup(D, t);
+            if (D.err) return;
+            if (rl.found) { found = true; at_root = true; qt = rl.tgt; plen = 0; root_slot = rl.slot; }
+            else {
+                if (D.lane == 0) D.root[rl.slot] = make_uint2(t, c | (k == 1 ? SAM_FLAG : 0u));
+                __syncwarp();
+                D.root_deg++;
+            }
+            break;
+        }
+        lk = lookup_state(D, p, t);
+        if (lk.found) { found = true; qt = lk.tgt; plen = lk.len; break; }
+        insert_edge(D, p, lk, t, c);                   // len[p] + 1 < k: not solid
+        if (D.err) return;
+        p = lk.link;
+        if (--guard < 0) { D.err = SAM_SEQ_WALK_LIMIT; return; }
+    }
+
+    if (!found) {                                      // walked past the root
+        s2 = 0; l2 = 0;
+    } else {
+        const uint32_t q = qt & SAM_IDMASK;
+        if (qt & SAM_FLAG) {                           // len[p] + 1 == len[q]
+            s2 = q; l2 = plen + 1;
+        } else {
+            // clone q as cl with len[p] + 1
+            const uint32_t cl = D.n_states;
+            ensure_rec(D, cl);
+            if (D.err) return;
+            D.n_states = cl + 1;
+            uint4* rq = rec_ptr(D, q);
+            const uint4 qa = rq[0], qb = rq[1];
+            uint4 nb;
+            if (qa.w <= 2) {
+                nb = make_uint4(qb.x, qb.y & SAM_IDMASK, qb.z, qb.w & SAM_IDMASK);   // copies are never solid
+            } else {
+                uint32_t noff = alloc_block(D, qb.y);
+                if (D.err) return;
+                const uint2* ob = blk_ptr(D, qb.x);
+                uint2* nbk = blk_ptr(D, noff);
+                for (uint32_t i = D.lane; i < qa.w; i += 32) { uint2 e = ob[i]; e.y &= SAM_IDMASK; nbk[i] = e; }
+                nb = make_uint4(noff, qb.y, 0, 0);
+            }
+            uint4* rc = rec_ptr(D, cl);
+            if (D.lane == 0) {
+                rc[0] = make_uint4(plen + 1, qa.y, qa.z, qa.w);      // link[q], min_endpos[q], deg[q]
+                rc[1] = nb;
+            }
+            __syncwarp();
+            // redirect p and the states above it whose t-transition is q
+            if (at_root) {
+                if (D.lane == 0) D.root[root_slot].y = cl | SAM_FLAG;
+            } else {
+                uint32_t* rw = reinterpret_cast<uint32_t*>(rec_ptr(D, p));
+                if (D.lane == 0) {
+                    if (lk.deg <= 2) rw[5 + 2 * lk.idx] = cl | SAM_FLAG;
+                    else blk_ptr(D, lk.b0)[lk.idx].y = cl | SAM_FLAG;
+                }
+                uint32_t pp = lk.link;
+                int g2 = (int)plen + 2;
+                for (;;) {
+                    if (pp == 0) {
+                        RootLook r2 = root_lookup(D, t);
+                        if (D.err) return;
+                        if (r2.found && (r2.tgt & SAM_IDMASK) == q) {
+                            if (D.lane == 0) D.root[r2.slot].y = cl;
+                        }
+                        break;
+                    }
+                    Look l2k = lookup_state(D, pp, t);
+                    if (!l2k.found) { D.err = SAM_SEQ_WALK_LIMIT; return; }   // every state up the chain has t
+                    if ((l2k.tgt & SAM_IDMASK) != q) break;
+                    uint32_t* rw2 = reinterpret_cast<uint32_t*>(rec_ptr(D, pp));
+                    if (D.lane == 0) {
+                        if (l2k.deg <= 2) rw2[5 + 2 * l2k.idx] = cl;
+                        else blk_ptr(D, l2k.b0)[l2k.idx].y = cl;
+                    }
+                    pp = l2k.link;
+                    if (--g2 < 0) { D.err = SAM_SEQ_WALK_LIMIT; return; }
+                }
+            }
+            if (D.lane == 0) reinterpret_cast<uint32_t*>(rq)[1] = cl;        // link[q] = cl
+            __syncwarp();
+            s2 = cl; l2 = plen + 1;
+        }
+    }
+    if (D.lane == 0) D.text[ntok] = (int32_t)t;
+    last = c; ntok = k;
+}
+
+// ------------------------------------------------------------------ the kernel
+__global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ StepArgs A) {
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __shared__ int32_t sh_l[2], sh_s[2], sh_dl[2], sh_err[2];
+
+    uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const uint32_t cw = cb[lane];                       // control words 0..31
+    int status = (int)__shfl_sync(FULL, cw, CB_STATUS);
+    const uint32_t ntok0 = __shfl_sync(FULL, cw, CB_NTOK);
+    const int m = A.counts[b];
+    const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
+    const int L = A.L;
+    __syncthreads();          // both warps hold the slot's state as it was before either writes any of it
+
+    // validate the whole step before any state changes (both warps reach the same verdict)
+    bool fresh_fail = false;
+    if (status == 0) {
+        if (m < 0 || m > A.stride) status = SAM_SEQ_BAD_COUNT;
+        else if ((int64_t)ntok0 + m > A.W.max_seq_len) status = SAM_SEQ_CAPACITY;
+        else {
+            const int vocab = A.has_static ? A.S.vocab : A.W.vocab;
+            bool bad = false;
+            for (int base = 0; base < m; base += 32) {
+                int i = base + lane;
+                if (i < m) { int t = toks[i]; bad |= (t < 0 || t >= vocab); }
+            }
+            if (__any_sync(FULL, bad)) status = SAM_SEQ_BAD_TOKEN;
+        }
+        fresh_fail = status != 0;
+    }
+    if (status != 0) {
+        if (warp == 0) {
+            if (fresh_fail && lane == 0) cb[CB_STATUS] = (uint32_t)status;
+            for (int j = lane; j < L; j += 32) A.draft_tokens[(size_t)b * L + j] = -1;
+            if (lane == 0) {
+                A.draft_len[b] = 0; A.match_len[2 * b] = 0; A.match_len[2 * b + 1] = 0; A.source[b] = 0;
+                if (A.state) { A.state[2 * b] = 0; A.state[2 * b + 1] = 0; }
+                A.status[b] = status;
+            }
+        }
+        return;
+    }
+
+    int32_t d[MAX_DRAFT_REGS] = {-1, -1, -1, -1};
+    int32_t my_l = 0, my_s = 0, my_dl = 0;
+    int err = 0;
+
+    if (warp == 0) {
+        // ---------------- static automaton: Transfer per token ----------------
+        if (A.has_static) {
+            uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
+            int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
+            for (int base = 0; base < m && !err; base += 32) {
+                const int i = base + lane;
+                uint32_t tk = 0, re = SAM_NONE;
+                if (i < m) { tk = (uint32_t)toks[i]; re = __ldg(A.S.root_row + tk); }
+                const int cnt = min(32, m - base);
+                for (int j = 0; j < cnt && !err; j++)
+                    static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err);
+            }
+            if (m > 0 && lane == 0 && !err) { cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf; }
+            my_l = l; my_s = (int32_t)s;
+            if (l > 0 && !err) {
+                const int64_t e = (int64_t)__ldg(A.S.rec + 2 * (size_t)s).z;       // min_endpos
+                int64_t room = A.S.n_tokens - e;
+                my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
+                gather_draft<true>(A.S.corpus, e, my_dl, L, lane, d);
+            }
+        }
+    } else {
+        // ---------------- dynamic automaton: Expand per token ----------------
+        Dyn D;
+        D.pool = A.W.pool;
+        D.root = A.W.root_tab + (size_t)b * A.W.root_cap;
+        D.text = A.W.text + (size_t)b * A.W.text_stride;
+        D.pool_hdr = A.W.pool_hdr; D.free_stack = A.W.free_stack; D.slab_owner = A.W.slab_owner;
+        D.cb = cb;
+        D.tab = cb[CB_SLABTAB + lane];
+        D.n_rec_slabs = __shfl_sync(FULL, cw, CB_NRECSLABS);
+        D.n_states = __shfl_sync(FULL, cw, CB_NSTATES);
+        D.blk_cur = __shfl_sync(FULL, cw, CB_BLK_CUR);
+        D.blk_end = __shfl_sync(FULL, cw, CB_BLK_END);
+        D.root_deg = __shfl_sync(FULL, cw, CB_ROOTDEG);
+        D.root_bmask = (uint32_t)(A.W.root_cap / SAM_ROOT_BUCKET) - 1;
+        D.slab_shift = A.W.slab_shift; D.rps_shift = A.W.slab_shift - 5;
+        D.seq = b; D.lane = lane; D.err = 0;
+        uint32_t last = __shfl_sync(FULL, cw, CB_LAST), ntok = ntok0;
+        uint32_t s2 = __shfl_sync(FULL, cw, CB_S2), l2 = __shfl_sync(FULL, cw, CB_L2);
+        if (D.n_states == 0) D.n_states = 1;            // the root exists implicitly (no record is read for it)
+
+        for (int base = 0; base < m && !D.err; base += 32) {
+            const int i = base + lane;
+            uint32_t tk = 0;
+            if (i < m) tk = (uint32_t)toks[i];
+            const int cnt = min(32, m - base);
+            for (int j = 0; j < cnt && !D.err; j++)
+                dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2);
+        }
+        err = D.err;
+        if (m > 0 && !err) {
+            // the newest state's record, without a transition yet
+            uint4* rl = rec_ptr(D, last);
+            if (lane == 0) {
+                rl[0] = make_uint4(ntok, s2, ntok, 0);
+                rl[1] = make_uint4(0, 0, 0, 0);
+                cb[CB_NTOK] = ntok; cb[CB_NSTATES] = D.n_states; cb[CB_LAST] = last;
+                cb[CB_S2] = s2; cb[CB_L2] = l2; cb[CB_BLK_CUR] = D.blk_cur; cb[CB_BLK_END] = D.blk_end;
+                cb[CB_NRECSLABS] = D.n_rec_slabs; cb[CB_ROOTDEG] = D.root_deg;
+            }
+            __syncwarp();
+        }
+        my_l = (int32_t)l2; my_s = (int32_t)s2;
+        if (l2 > 0 && !err) {
+            const int64_t e = (int64_t)rec_ptr(D, s2)[0].z;                       // min_endpos
+            int64_t room = (int64_t)ntok - e;
+            my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
+            gather_draft<false>(D.text, e, my_dl, L, lane, d);
+        }
+    }
+
+    if (lane == 0) { sh_l[warp] = my_l; sh_s[warp] = my_s; sh_dl[warp] = my_dl; sh_err[warp] = err; }
+    __syncthreads();
+    const int any_err = sh_err[0] ? sh_err[0] : sh_err[1];
+    const int l1 = sh_l[0], l2v = sh_l[1];
+    const bool use_static = A.has_static && l1 > l2v + A.W.l_bias;        // Section 3.2
+    const int lsel = use_static ? l1 : l2v;
+    const int need = A.W.min_match > 1 ? A.W.min_match : 1;
+    const int src = (any_err || lsel < need) ? SAM_SRC_NONE : (use_static ? SAM_SRC_STATIC : SAM_SRC_DYNAMIC);
+    const int winner = src == SAM_SRC_DYNAMIC ? 1 : 0;
+
+    if (warp == winner) {
+#pragma unroll
+        for (int r = 0; r < MAX_DRAFT_REGS; r++) {
+            int j = r * 32 + lane;
+            if (j < L) A.draft_tokens[(size_t)b * L + j] = (src == SAM_SRC_NONE) ? -1 : d[r];
+        }
+    }
+    if (warp == 0 && lane == 0) {
+        if (any_err) cb[CB_STATUS] = (uint32_t)any_err;
+        A.draft_len[b] = src == SAM_SRC_NONE ? 0 : sh_dl[winner];
+        A.match_len[2 * b] = any_err ? 0 : l1;
+        A.match_len[2 * b + 1] = any_err ? 0 : l2v;
+        A.source[b] = src;
+        if (A.state) { A.state[2 * b] = any_err ? 0 : sh_s[0]; A.state[2 * b + 1] = any_err ? 0 : sh_s[1]; }
+        A.status[b] = any_err;
+    }
+}
+
+}  // namespace
+
+int sam_launch_step(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
+                    int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
+                    int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream) {
+    StepArgs A;
+    A.has_static = b->st != nullptr;
+    if (b->st) A.S = b->st->view;
+    else { A.S = SamStaticView(); A.S.vocab = b->view.vocab; }
+    A.W = b->view;
+    A.new_tokens = new_tokens; A.stride = stride; A.counts = counts; A.L = L;
+    A.draft_tokens = draft_tokens; A.draft_len = draft_len; A.match_len = match_len;
+    A.source = source; A.state = state; A.status = status;
+    sam_step_kernel<<<b->view.batch, 64, 0, stream>>>(A);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
+    return SAM_OK;
+}

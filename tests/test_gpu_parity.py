@@ -1,0 +1,209 @@
+"""GPU parity: the CUDA library against the CPU oracle, bit for bit, through the C ABI."""
+import os
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+from _parity import assert_dynamic_automata_equal, assert_same, gpu_run, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "abcbc_automaton.txt")
+
+
+@pytest.fixture(scope="module")
+def P():
+    import torch
+    assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
+    import paper_2411_10666_b200 as pkg
+    pkg.lib()
+    return pkg
+
+
+def _steps_from_text(x, rng, kmax):
+    """Split a token list into (new_tokens [S,1,K], counts [S,1])."""
+    rows, cnts, k = [], [], 0
+    while k < len(x):
+        m = min(rng.randint(0, kmax), len(x) - k)
+        rows.append(x[k:k + m] + [-1] * (kmax - m))
+        cnts.append(m)
+        k += m
+    return np.array(rows, dtype=np.int32).reshape(-1, 1, kmax), np.array(cnts, dtype=np.int32).reshape(-1, 1)
+
+
+def test_abcbc_golden(P):
+    T = np.array([0, 1, 2, 1, 2], dtype=np.int32)
+    st = P.StaticSam.build(T, 3)
+    tb = P.binding.sam_static_tables(st.handle)
+    rows = [l.split() for l in open(GOLDEN) if l[0].isdigit()]
+    for f in rows:
+        sid = int(f[0])
+        assert (tb["length"][sid], tb["link"][sid], tb["min_endpos"][sid]) == (int(f[1]), int(f[2]), int(f[3]))
+        exp = {} if f[4] == "-" else {int(a): int(b) for a, b in (e.split(">") for e in f[4].split(","))}
+        assert P.binding.sam_static_state(st.handle, sid)["next"] == exp
+    # static stream B,C,B,A with a disabled dynamic side cannot be had; use l_bias=0 rows where static wins
+    trans = [l.split() for l in open(GOLDEN) if l.startswith("T ")]
+    dyn = [l.split() for l in open(GOLDEN) if l.startswith("D ")]
+    lst = lambda s: [] if s == "-" else [int(v) for v in s.split(",")]
+    toks = np.array([[[int(f[1])]] for f in trans], dtype=np.int32)
+    res, _ = gpu_run(P, st, 3, np.zeros((1, 0), np.int32), toks, np.ones((len(trans), 1), np.int32), 3, 16)
+    for i, f in enumerate(trans):
+        assert res["state"][i, 0, 0] == int(f[2]) and res["match_len"][i, 0, 0] == int(f[3])
+        if res["source"][i, 0] == 1:
+            d = lst(f[6])
+            assert res["draft_tokens"][i, 0, :len(d)].tolist() == d and res["draft_len"][i, 0] == len(d)
+    assert (res["source"][:, 0] == 1).sum() >= 3
+    toks = np.array([[[int(f[1])]] for f in dyn], dtype=np.int32)
+    res, batch = gpu_run(P, None, 3, np.zeros((1, 0), np.int32), toks, np.ones((len(dyn), 1), np.int32), 3, 16)
+    for i, f in enumerate(dyn):
+        assert res["state"][i, 0, 1] == int(f[2]) and res["match_len"][i, 0, 1] == int(f[3])
+        d = lst(f[5])
+        assert res["draft_len"][i, 0] == len(d) and res["draft_tokens"][i, 0, :len(d)].tolist() == d
+    d = batch.dump(0, 16, 16)
+    assert d["n_states"] == 8 and d["n_edges"] == 9
+    for f in rows:
+        sid = int(f[0])
+        assert (d["length"][sid], d["link"][sid], d["min_endpos"][sid]) == (int(f[1]), int(f[2]), int(f[3]))
+
+
+def _rand_text(rng, n, vocab, copy_p):
+    x = []
+    while len(x) < n:
+        if x and rng.random() < copy_p:
+            s = rng.randrange(len(x))
+            x.extend(x[s:s + rng.randint(1, 20)])
+        else:
+            x.append(rng.randrange(vocab))
+    return x[:n]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_small_cases_all_outputs_and_automata(P, seed):
+    rng = random.Random(100 + seed)
+    for case in range(6):
+        vocab = rng.choice([2, 3, 5, 50, 1000])
+        N = rng.choice([1, 7, 200, 3000])
+        n = rng.choice([1, 33, 257, 900])
+        L = rng.choice([1, 5, 32, 33, 128])
+        kmax = rng.choice([1, 4, 40])
+        l_bias, min_match = rng.choice([(0, 1), (0, 0), (2, 1), (0, 3), (5, 5)])
+        corpus = np.array(_rand_text(rng, N, vocab, 0.3), dtype=np.int32)
+        B = rng.choice([1, 3])
+        texts = []
+        for b in range(B):
+            x = _rand_text(rng, n, vocab, 0.4)
+            if N > 20 and rng.random() < 0.7:                # splice corpus spans in
+                for _ in range(3):
+                    s = rng.randrange(N); ln = rng.randint(2, 40); at = rng.randrange(n)
+                    x[at:at + ln] = corpus[s:s + ln].tolist()
+                x = x[:n]
+            texts.append(x + [0] * (n - len(x)))
+        # a common step schedule for all slots
+        rows, cnts, k = [], [], 0
+        while k < n:
+            m = min(rng.randint(0, kmax), n - k)
+            rows.append([t[k:k + m] + [-1] * (kmax - m) for t in texts])
+            cnts.append([m] * B)
+            k += m
+        nt = np.array(rows, dtype=np.int32).reshape(len(rows), B, kmax)
+        ct = np.array(cnts, dtype=np.int32).reshape(len(rows), B)
+        empty = np.zeros((B, 0), np.int32)
+        st = P.StaticSam.build(corpus, vocab)
+        ref, ob, _ = oracle_run(corpus, vocab, empty, nt, ct, L, n, l_bias, min_match)
+        got, batch = gpu_run(P, st, vocab, empty, nt, ct, L, n, l_bias, min_match)
+        assert_same(got, ref, "seed %d case %d" % (seed, case))
+        assert_dynamic_automata_equal(batch, ob, range(B), n)
+        assert (got["status"] == 0).all()
+
+
+def test_adversarial_sequences(P):
+    n = 1500
+    cases = [
+        [0] * n,
+        [0] + [1] * (n - 1),
+        [0] + [1] * (n - 2) + [2],
+        [i % 7 for i in range(n)],
+        [v for i in range(n // 2) for v in (0, 1 + i)],       # a state with n/2 successors: block growth
+        list(range(n)),
+        [(i * i) % 11 for i in range(n)],
+        [v for i in range(n // 3) for v in (0, 1, 2 + i)],
+    ]
+    rng = random.Random(5)
+    for x in cases:
+        vocab = max(x) + 1
+        nt, ct = _steps_from_text(x, rng, 64)
+        empty = np.zeros((1, 0), np.int32)
+        ref, ob, _ = oracle_run(None, vocab, empty, nt, ct, 8, n)
+        got, batch = gpu_run(P, None, vocab, empty, nt, ct, 8, n)
+        assert_same(got, ref)
+        assert_dynamic_automata_equal(batch, ob, [0], n)
+
+
+CASES = {
+    # name: (spec key, corpus_len, batch, prompt_len, gen_len) — same recipes, smaller sizes
+    "tiny_full": ("tiny", None, None, None, None),
+    "c2_small": ("c2", 400_000, 16, 512, 700),
+    "c3_small": ("c3", 600_000, 24, 600, 900),
+    "c4_small": ("c4", 200_000, 32, 1500, 700),
+    "c5_small": ("c5", 500_000, 96, 500, 500),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_workload_recipes(P, name):
+    key, N, B, pl, gl = CASES[name]
+    spec = W.scaled(W.SPECS[key], N, B, pl, gl)
+    w = W.make(spec)
+    L = spec.draft_len
+    msl = spec.prompt_len + spec.gen_len
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=4)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    assert_same(got, ref, name)
+    assert (got["status"] == 0).all()
+    assert_dynamic_automata_equal(batch, ob, [0, spec.batch - 1], msl)
+    assert (got["source"] == 1).any() or key == "c4"
+    assert (got["source"] == 2).any()
+    info = st.info
+    assert info.n_states == S.n_states and info.n_transitions == S.n_transitions
+
+
+def test_c2_full_size_bench_configuration(P):
+    """Config 2 at full size, launched exactly as the benchmark launches it (prefill step, then one
+    launch per decoding step through sam_run_steps): every output of every step equals the oracle."""
+    spec = W.SPECS["c2"]
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=8)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    assert_same(got, ref, "c2 full")
+    assert st.info.n_states == S.n_states
+    # self-certifying sample: the reported match is a suffix occurrence at the reported end position
+    rng = random.Random(2)
+    tb = P.binding.sam_static_tables(st.handle)
+    pos = np.full(spec.batch, spec.prompt_len) + np.cumsum(w.counts, axis=0)
+    for _ in range(300):
+        s = rng.randrange(w.n_steps); b = rng.randrange(spec.batch)
+        k = int(pos[s, b]); x = w.seqs[b, :k]
+        l1 = int(got["match_len"][s + 1, b, 0]); e1 = int(tb["min_endpos"][got["state"][s + 1, b, 0]])
+        assert (w.corpus[e1 - l1:e1] == x[k - l1:]).all()
+        if got["source"][s + 1, b] == 1:
+            dl = int(got["draft_len"][s + 1, b])
+            assert (got["draft_tokens"][s + 1, b, :dl] == w.corpus[e1:e1 + dl]).all()
+
+
+@pytest.mark.skipif(os.environ.get("SAMDRAFT_FULL") != "1", reason="minutes and tens of GB: set SAMDRAFT_FULL=1")
+@pytest.mark.parametrize("key", ["c4", "c3", "c5"])
+def test_full_size_configs(P, key):
+    spec = W.SPECS[key]
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=os.cpu_count())
+    assert_same(got, ref, key)
+    assert st.info.n_states == S.n_states and st.info.n_transitions == S.n_transitions
