@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the batched suffix-automaton draft-retrieval step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
+
+A "step" is one `sam_step` over the whole batch: every slot feeds its accepted tokens of that
+decoding step through the static automaton (Transfer) and its own dynamic automaton
+(Transfer + Expand), the source is chosen and the draft is read.  The prompt prefill and W
+warm-up steps run untimed; then exactly K consecutive decoding steps of the schedule are timed
+with CUDA events (one kernel launch per step).  The K-step region is repeated from an identical
+state (reset, prefill, warm-up, L2 flush) until a few seconds have passed so that clock samples
+exist; the reported value is the median repeat.  One JSON line is printed by rank 0.
+
+Under torchrun each rank owns a contiguous shard of a batch that is N times larger (weak scaling,
+the static automaton replicated, no collective on the data path); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+METRIC = "sam_sequence_steps_per_sec"
+UNIT = "sequence-steps/s"
+
+# Algorithmic bytes per sequence-step of the generation phase: what the method itself must read
+# and write, from the CPU oracle's operation counters (python -m oracle.count_ops <workload>):
+# 32 B per Transfer move, per walk-insert (+8 B edge), per clone (x2), per redirect (+4 B);
+# 32 B new state + 8 B links + 4 B text per token; per step two 32-B records, the drafted tokens
+# and the input and output rows.
+ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 900.0, "c4": 1374.8, "c5": 1000.0}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(W.SPECS))
+    ap.add_argument("--min-seconds", type=float, default=2.5, help="keep repeating the timed region this long")
+    ap.add_argument("--max-repeats", type=int, default=300)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-probes", action="store_true")
+    return ap.parse_args()
+
+
+def dist_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of one GPU while the timed regions run."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="samclk_", suffix=".csv")
+            self.f = os.fdopen(fd, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def shard_workload(spec: W.Spec, rank: int, world: int):
+    """Weak scaling: the global batch is `world` times the recipe's batch; this rank's shard."""
+    big = W.scaled(spec, batch=spec.batch * world)
+    corpus = W.make_corpus(big)
+    seqs, counts, new_tokens = W.make_sequences(big, corpus, rank, world)
+    return big, corpus, seqs, counts, new_tokens
+
+
+def reduce_max_sum(local_ms: float, local_units: int, world: int):
+    """(max over ranks of the time, sum over ranks of the units) — the only cross-rank exchange."""
+    if world == 1:
+        return local_ms, local_units
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([local_units], dtype=torch.int64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(u.item())
+
+
+def run_oracle_timed(spec, corpus, seqs, counts, new_tokens, steps_lo, steps_hi, threads, static=None):
+    """Time the CPU oracle on decoding steps [steps_lo, steps_hi) after an untimed build, prefill
+    and the steps before steps_lo.  Returns (seconds, sequence-steps, draft tokens, automaton)."""
+    import oracle
+    S = static if static is not None else oracle.Sam(corpus)
+    B, L = seqs.shape[0], spec.draft_len
+    ob = oracle.Batch(S, corpus, B, spec.vocab, spec.prompt_len + spec.gen_len)
+    ob.step(np.ascontiguousarray(seqs[:, :spec.prompt_len]), np.full(B, spec.prompt_len, dtype=np.int32), L, threads)
+    if steps_lo > 0:
+        ob.run(new_tokens[:steps_lo], counts[:steps_lo], L, threads)
+    c0 = ob.counters()
+    t0 = time.perf_counter()
+    ob.run(new_tokens[steps_lo:steps_hi], counts[steps_lo:steps_hi], L, threads)
+    dt = time.perf_counter() - t0
+    c1 = ob.counters()
+    ob.close()
+    return dt, c1["seq_steps"] - c0["seq_steps"], c1["draft_tokens"] - c0["draft_tokens"], S
+
+
+def main_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    spec = W.SPECS[args.workload]
+    corpus = W.make_corpus(spec)
+    seqs, counts, new_tokens = W.make_sequences(spec, corpus)
+    K = min(args.steps, counts.shape[0] - args.warmup)
+    threads = os.cpu_count() or 1
+    dt, units, drafts, _ = run_oracle_timed(spec, corpus, seqs, counts, new_tokens, args.warmup, args.warmup + K, threads)
+    value = units / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": K, "warmup": args.warmup, "ms_per_step": dt * 1e3 / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "prompt_len": spec.prompt_len,
+                   "gen_len": spec.gen_len, "draft_len": spec.draft_len, "corpus_tokens": spec.corpus_len},
+        "draft_tokens_per_sec": drafts / dt,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": "decoding steps [%d, %d) of %s, all %d sequences, OpenMP over sequences; "
+                                   "static build and prefill untimed" % (args.warmup, args.warmup + K, spec.name, spec.batch)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main_ours(args):
+    import torch
+    rank, world, local_rank = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the retrieval path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+    import paper_2411_10666_b200 as P
+    sd = P.binding
+    P.lib()
+
+    base = W.SPECS[args.workload]
+    spec, corpus, seqs, counts, new_tokens = shard_workload(base, rank, world)
+    B, L = seqs.shape[0], spec.draft_len
+    msl = spec.prompt_len + spec.gen_len
+    Wm = args.warmup
+    K = min(args.steps, counts.shape[0] - Wm)
+    assert K >= 1 and Wm >= 3, "need at least 3 warm-up steps and 1 timed step"
+
+    t0 = time.perf_counter()
+    st = P.StaticSam.build(corpus, spec.vocab, device=local_rank)
+    build_s = time.perf_counter() - t0
+    info = st.info
+    batch = P.Batch(st, B, msl, max_draft_len=L, max_host_stride=spec.accept_max)
+    dev = batch.device
+    prompts = torch.from_numpy(np.ascontiguousarray(seqs[:, :spec.prompt_len])).to(dev)
+    pcount = torch.full((B,), spec.prompt_len, dtype=torch.int32, device=dev)
+    nt_dev = torch.from_numpy(new_tokens).to(dev)
+    ct_dev = torch.from_numpy(counts).to(dev)
+    out = P.StepOutputs(B, L, dev)
+    flush = torch.empty(288 << 20, dtype=torch.uint8, device=dev)      # larger than the 126 MB L2
+
+    def prepare():
+        batch.reset()
+        batch.step(prompts, pcount, L, out)
+        batch.run_steps(nt_dev[:Wm], ct_dev[:Wm], L, per_step=False, out=out)
+        flush.zero_()
+
+    units = int((counts[Wm:Wm + K] > 0).sum())
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # prefill throughput, reported separately (not part of the headline)
+    batch.reset()
+    torch.cuda.synchronize()
+    e0.record()
+    batch.step(prompts, pcount, L, out)
+    e1.record()
+    torch.cuda.synchronize()
+    prefill_ms = e0.elapsed_time(e1)
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    times = []
+    t_start = time.perf_counter()
+    while True:
+        prepare()
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        e0.record()
+        batch.run_steps(nt_dev[Wm:Wm + K], ct_dev[Wm:Wm + K], L, per_step=False, out=out)
+        e1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        times.append(e0.elapsed_time(e1))
+        elapsed = time.perf_counter() - t_start
+        stop = len(times) >= 3 and (elapsed >= args.min_seconds or len(times) >= args.max_repeats)
+        if world > 1:                                                   # all ranks stop together
+            flag = torch.tensor([1 if stop else 0], device=dev)
+            torch.distributed.all_reduce(flag, op=torch.distributed.ReduceOp.MAX)
+            stop = bool(flag.item())
+        if stop:
+            break
+    status_ok = bool((out.status == 0).all().item())
+
+    # end to end through the host-array call: pinned inputs, H2D + step + D2H + sync every step
+    nt_pin = torch.from_numpy(new_tokens).pin_memory()
+    ct_pin = torch.from_numpy(counts).pin_memory()
+    mk = lambda *s: torch.empty(s, dtype=torch.int32).pin_memory()
+    ho = [mk(B, L), mk(B), mk(B, 2), mk(B), mk(B, 2), mk(B)]
+    e2e_times = []
+    for _ in range(3):
+        prepare()
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        t1 = time.perf_counter()
+        for s in range(Wm, Wm + K):
+            sd.sam_step_host(batch.handle, nt_pin[s], spec.accept_max, ct_pin[s], L, *ho)
+        torch.cuda.synchronize()
+        e2e_times.append((time.perf_counter() - t1) * 1e3)
+    clocks = sampler.stop() if sampler else None
+
+    # draft tokens per second: count drafted tokens of every timed step once (untimed pass)
+    prepare()
+    per = batch.run_steps(nt_dev[Wm:Wm + K], ct_dev[Wm:Wm + K], L, per_step=True)
+    active = ct_dev[Wm:Wm + K] > 0
+    draft_tokens = int((per.draft_len * active).sum().item())
+    accepted_tokens = int(counts[Wm:Wm + K].sum())
+    torch.cuda.synchronize()
+
+    ms_local = statistics.median(times)
+    ms, units_all = reduce_max_sum(ms_local, units, world)
+    e2e_ms, _ = reduce_max_sum(statistics.median(e2e_times), units, world)
+    _, drafts_all = reduce_max_sum(0.0, draft_tokens, world)
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return 0
+
+    value = units_all / (ms * 1e-3)
+    launch_us = ms_local * 1e3 / K
+    algo_b = ALGO_BYTES[base.name]
+    achieved = algo_b * (units / K) / (launch_us * 1e-6) / 1e9          # GB/s of one launch on this rank
+    peak_src = "fallback"
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        peak, peak_src = float(peaks["hbm_gbs"]), "measured"
+    except Exception:
+        peak = 6650.0
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": peak_src + " stream copy",
+                "kernel": "sam_step_kernel", "launch_us": launch_us,
+                "algorithmic_bytes_per_sequence_step": algo_b,
+                "sequence_steps_per_launch": units / K}
+
+    if not args.no_probes:
+        # the random-access denominators, measured now on a buffer the size of the static store
+        fp = min(max(int(info.device_bytes), 256 << 20), 8 << 30)
+        buf = torch.empty(fp, dtype=torch.uint8, device=dev)
+        rnd = {}
+        for g in (32, 64, 128):
+            gbps, mreq = sd.sam_probe_random_read(buf, g, iters=3)
+            rnd[str(g)] = {"GB/s": round(gbps, 1), "Mreq/s": round(mreq, 1)}
+        chains = 2 * B
+        ns1 = sd.sam_probe_chase(buf, 20000, chains=1)
+        nsc = sd.sam_probe_chase(buf, 20000, chains=chains)
+        del buf
+        roofline["random_read"] = rnd
+        roofline["frac_of_random_32B"] = achieved / rnd["32"]["GB/s"]
+        roofline["dependent_load_ns"] = {"1_chain": round(ns1, 1), "%d_chains" % chains: round(nsc, 1)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": base.name, "batch_per_gpu": B, "global_batch": B * world,
+                   "prompt_len": spec.prompt_len, "gen_len": spec.gen_len, "draft_len": L,
+                   "corpus_tokens": spec.corpus_len, "vocab": spec.vocab,
+                   "static_states": int(info.n_states), "static_bytes": int(info.device_bytes),
+                   "parallelism": "batch-sharded x%d, static automaton replicated" % world,
+                   "l2": "L2 flushed (288 MB write) before each timed region; static store %.2f GB exceeds the 126 MB L2; "
+                         "per-sequence automata stay cache-warm between consecutive steps" % (info.device_bytes / 1e9),
+                   "repeats": len(times), "timing": "median of repeats, CUDA events, max over ranks"},
+        "draft_tokens_per_sec": drafts_all / (ms * 1e-3),
+        "accepted_tokens_per_sec": accepted_tokens * world / (ms * 1e-3),
+        "best_ms_per_step": min(times) / K,
+        "prefill_tokens_per_sec": B * spec.prompt_len / (prefill_ms * 1e-3),
+        "static_build_seconds": build_s,
+        "status_all_ok": status_ok,
+        "e2e": {"value": units_all / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": B * spec.accept_max * 4 + B * 4, "d2h_bytes_per_step": B * (L + 7) * 4,
+                "ms_per_step": e2e_ms / K, "api": "sam_step_host"},
+        "gpu_launches": K,
+        "clocks": clocks,
+        "roofline": roofline,
+    }
+
+    if world == 1 and not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        dt, u, _, S = run_oracle_timed(base, corpus, seqs, counts, new_tokens, Wm, Wm + K, cores)
+        dt1, u1, _, _ = run_oracle_timed(base, corpus, seqs, counts, new_tokens, Wm, Wm + K, 1, static=S)
+        line["cpu_baseline"] = {"value": u / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "single_thread_value": u1 / dt1,
+                                "sample": "the same %d decoding steps x %d sequences (%d sequence-steps), OpenMP over "
+                                          "sequences; static build and prefill untimed" % (K, B, u)}
+    print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    sys.exit(main_reference(a) if a.impl == "reference" else main_ours(a))
