@@ -215,6 +215,42 @@ int sam_batch_pool_info(sam_batch_t* b, int64_t* total_slabs, int64_t* free_slab
 /* Forget the batch.  The workspace is the caller's and is not freed. */
 void sam_batch_destroy(sam_batch_t* b);
 
+/* ---- retrieval without any allocation ------------------------------------------------------ */
+
+/* (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * One-shot retrieval for callers that cannot allocate device memory: a drafting hook that runs
+ * inside an inference server which has already given the device's free memory to its own KV-cache
+ * pool, or any component held to a "no allocation after start-up" rule.  Such a caller cannot
+ * provide the workspace sam_batch_create needs, so this call keeps the per-sequence automata in a
+ * fixed scratch array that is part of the library image: sam_noalloc_capacity_bytes() bytes
+ * (8 MiB), resident on every GPU that loads the library until the process exits.
+ *
+ * Semantics: exactly sam_batch_create on an empty batch of `batch` slots with max_seq_len = stride,
+ * followed by one sam_step — each slot i starts EMPTY, is fed tokens_dev[i, 0..counts_dev[i]) (its
+ * whole text so far: prompt plus accepted tokens) and reports the draft, lengths, source, states
+ * and status exactly as sam_step does.  Nothing persists between calls.
+ *   st may be NULL (then `vocab` gives the token range and l1 = 0); otherwise vocab is ignored.
+ *   tokens_dev device int32 [batch, stride]; counts_dev device int32 [batch]; outputs as sam_step
+ *   (state_dev may be NULL); l_bias and min_match as in sam_batch_opts_t; L in 1..128.
+ * Limits and errors: the layout for (batch, stride) must fit the scratch array, otherwise LIMIT is
+ * returned and nothing is launched (for scale: 16 slots of 1024 tokens need about 3.5 MiB); ARG for
+ * null pointers or out-of-range sizes; CUDA if the runtime fails.
+ * The call makes no cudaMalloc / cudaFree / pinned-host allocation.  The first call on a device
+ * looks up the array's device address (cudaGetSymbolAddress with that device current) and caches
+ * it; make that first call before any stream capture begins.  Work is enqueued on `stream` and is
+ * asynchronous.  All calls on a device share the one array and each call re-initialises it, so two
+ * calls whose kernels can overlap on the GPU (different streams, or other threads) race with each
+ * other: keep them on one stream or order them yourself. */
+int sam_retrieve_noalloc(const sam_static_t* st, int32_t vocab, int32_t batch,
+                         const int32_t* tokens_dev, int32_t stride, const int32_t* counts_dev,
+                         int32_t L, int32_t l_bias, int32_t min_match,
+                         int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,
+                         int32_t* source_dev, int32_t* state_dev, int32_t* status_dev, void* stream);
+
+/* Size of the built-in scratch array in bytes. */
+size_t sam_noalloc_capacity_bytes(void);
+
 /* ---- memory-system probes (the denominators of the random-access roofline) ---------------- */
 
 /* Independent uniformly random aligned reads of `granule` bytes (32, 64 or 128) over

@@ -74,6 +74,9 @@ SIGNATURES = {
                                c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "sam_batch_pool_info": (c_int, [c_void_p, POINTER(c_int64), POINTER(c_int64), c_void_p]),
     "sam_batch_destroy": (None, [c_void_p]),
+    "sam_retrieve_noalloc": (c_int, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32,
+                                     c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "sam_noalloc_capacity_bytes": (c_size_t, []),
     "sam_probe_random_read": (c_int, [c_void_p, c_size_t, c_int32, c_int32, c_void_p, POINTER(c_double), POINTER(c_double)]),
     "sam_probe_chase": (c_int, [c_void_p, c_size_t, c_int64, c_int32, c_void_p, POINTER(c_double)]),
     "sam_strerror": (c_char_p, [c_int]),
@@ -267,6 +270,17 @@ def sam_batch_pool_info(h, stream=None):
     tot, free = c_int64(), c_int64()
     _check(lib().sam_batch_pool_info(h, byref(tot), byref(free), _stream_ptr(stream)), "sam_batch_pool_info")
     return tot.value, free.value
+
+
+def sam_retrieve_noalloc(static_h, vocab, tokens, counts, L, l_bias, min_match,
+                         draft_tokens, draft_len, match_len, source, state, status, stream=None):
+    """One-shot retrieval over the library's built-in scratch array; allocates nothing."""
+    _check(lib().sam_retrieve_noalloc(static_h, vocab, tokens.shape[0], _dev_ptr(tokens, "tokens"), tokens.shape[1],
+                                      _dev_ptr(counts, "counts"), L, l_bias, min_match,
+                                      _dev_ptr(draft_tokens, "draft_tokens"), _dev_ptr(draft_len, "draft_len"),
+                                      _dev_ptr(match_len, "match_len"), _dev_ptr(source, "source"),
+                                      _dev_ptr(state, "state"), _dev_ptr(status, "status"), _stream_ptr(stream)),
+           "sam_retrieve_noalloc")
 
 
 def sam_probe_random_read(buf, granule: int, iters: int = 5, stream=None):

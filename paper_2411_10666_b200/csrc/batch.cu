@@ -150,6 +150,46 @@ __global__ void dump_kernel(SamBatchView W, int32_t slot, int32_t* hdr, int32_t*
 
 }  // namespace
 
+// ---- helpers for callers that bring their own memory for a short-lived batch ----------------
+
+// Lay a batch with these options out over `base` (device memory of at least *total bytes).
+int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBatchView* view,
+                  size_t* total, size_t* stage_words) {
+    WsLayout w;
+    int rc = plan(opts, &w);
+    if (rc) return rc;
+    if (total) *total = w.total;
+    if (stage_words) *stage_words = w.stage_words;
+    if (base && view) {
+        char* b = (char*)base;
+        view->pool_hdr = (int32_t*)(b + w.off_hdr);
+        view->ctrl = (uint32_t*)(b + w.off_ctrl);
+        view->free_stack = (int32_t*)(b + w.off_free);
+        view->slab_owner = (int32_t*)(b + w.off_owner);
+        view->reset_flag = (int32_t*)(b + w.off_reset);
+        view->text = (int32_t*)(b + w.off_text);
+        view->root_tab = (uint2*)(b + w.off_root);
+        view->stage = (int32_t*)(b + w.off_stage);
+        view->pool = (unsigned char*)(b + w.off_pool);
+        view->batch = opts->batch; view->max_seq_len = opts->max_seq_len; view->text_stride = w.text_stride;
+        view->root_cap = w.root_cap; view->slab_shift = w.slab_shift;
+        view->l_bias = opts->l_bias; view->min_match = opts->min_match;
+        view->vocab = vocab;
+        view->pool_slabs = w.pool_slabs;
+    }
+    return SAM_OK;
+}
+
+// Put every slot of the view into the empty state and fill the slab pool's free stack.
+int sam_launch_init(const SamBatchView& V, cudaStream_t s) {
+    init_pool_kernel<<<296, 256, 0, s>>>(V);
+    reset_slots_kernel<<<V.batch, 128, 0, s>>>(V, nullptr, V.batch);
+    clear_flags_kernel<<<(V.batch + 255) / 256, 256, 0, s>>>(V);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
+    return SAM_OK;
+}
+
 extern "C" int sam_batch_workspace_bytes(const sam_batch_opts_t* opts, size_t* out) {
     if (!opts || !out) return SAM_ERR_ARG;
     WsLayout w;

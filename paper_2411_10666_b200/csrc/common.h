@@ -52,3 +52,8 @@ static inline size_t sam_align_up(size_t x, size_t a) { return (x + a - 1) / a *
 int sam_launch_step(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
                     int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
                     int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream);
+
+// helpers implemented in batch.cu
+int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBatchView* view,
+                  size_t* total, size_t* stage_words);
+int sam_launch_init(const SamBatchView& V, cudaStream_t s);
