@@ -41,7 +41,7 @@ UNIT = "sequence-steps/s"
 # 32 B per Transfer move, per walk-insert (+8 B edge), per clone (x2), per redirect (+4 B);
 # 32 B new state + 8 B links + 4 B text per token; per step two 32-B records, the drafted tokens
 # and the input and output rows.
-ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1000.0}
+ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.1}
 
 
 def parse_args():

@@ -8,6 +8,8 @@
 
 namespace {
 
+constexpr size_t SAM_ZERO_COPY_MAX_BYTES = 256u << 10;   // larger host steps go through two DMA copies
+
 struct WsLayout {
     size_t off_hdr, off_ctrl, off_free, off_owner, off_reset, off_text, off_root, off_stage, off_pool, total;
     int32_t text_stride, root_cap, slab_shift, pool_slabs, max_host_stride;
@@ -244,8 +246,14 @@ extern "C" int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* 
 
     SamDeviceGuard guard(b->device);
     if (!guard.ok) { delete b; return SAM_ERR_CUDA; }
-    e = cudaHostAlloc((void**)&b->host_stage, w.stage_words * 4, cudaHostAllocDefault);
-    if (e != cudaSuccess) { sam_set_cuda_error(e); cudaGetLastError(); delete b; return SAM_ERR_NOMEM; }
+    e = cudaHostAlloc((void**)&b->host_stage, w.stage_words * 4, cudaHostAllocMapped);
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer((void**)&b->host_stage_dev, b->host_stage, 0);
+    if (e != cudaSuccess) {
+        sam_set_cuda_error(e); cudaGetLastError();
+        if (b->host_stage) cudaFreeHost(b->host_stage);
+        delete b;
+        return SAM_ERR_NOMEM;
+    }
     cudaStream_t s = (cudaStream_t)stream;
     init_pool_kernel<<<296, 256, 0, s>>>(V);
     reset_slots_kernel<<<V.batch, 128, 0, s>>>(V, nullptr, V.batch);
@@ -345,14 +353,25 @@ extern "C" int sam_step_host(sam_batch_t* b, const int32_t* new_tokens_host, int
     const size_t out_words = B * L + 7 * B;
     memcpy(hst, new_tokens_host, B * stride * 4);
     memcpy(hst + B * stride, counts_host, B * 4);
-    SAM_CUDA(cudaMemcpyAsync(dev, hst, in_words * 4, cudaMemcpyHostToDevice, s));
-    int32_t* o = dev + in_words;
-    rc = sam_launch_step(b, dev, stride, dev + B * stride, L, o, o + B * L, o + B * L + B, o + B * L + 3 * B,
-                         o + B * L + 4 * B, o + B * L + 6 * B, s);
-    if (rc) return rc;
     int32_t* ho = hst + in_words;
-    SAM_CUDA(cudaMemcpyAsync(ho, o, out_words * 4, cudaMemcpyDeviceToHost, s));
-    SAM_CUDA(cudaStreamSynchronize(s));
+    if ((in_words + out_words) * 4 <= SAM_ZERO_COPY_MAX_BYTES) {
+        // small steps: the kernel reads its inputs from, and writes its outputs to, the mapped host
+        // staging area directly; the bytes cross the bus inside the kernel instead of in two copies
+        int32_t* zd = b->host_stage_dev;
+        int32_t* zo = zd + in_words;
+        rc = sam_launch_step(b, zd, stride, zd + B * stride, L, zo, zo + B * L, zo + B * L + B, zo + B * L + 3 * B,
+                             zo + B * L + 4 * B, zo + B * L + 6 * B, s);
+        if (rc) return rc;
+        SAM_CUDA(cudaStreamSynchronize(s));
+    } else {
+        SAM_CUDA(cudaMemcpyAsync(dev, hst, in_words * 4, cudaMemcpyHostToDevice, s));
+        int32_t* o = dev + in_words;
+        rc = sam_launch_step(b, dev, stride, dev + B * stride, L, o, o + B * L, o + B * L + B, o + B * L + 3 * B,
+                             o + B * L + 4 * B, o + B * L + 6 * B, s);
+        if (rc) return rc;
+        SAM_CUDA(cudaMemcpyAsync(ho, o, out_words * 4, cudaMemcpyDeviceToHost, s));
+        SAM_CUDA(cudaStreamSynchronize(s));
+    }
     memcpy(draft_tokens_host, ho, B * L * 4);
     memcpy(draft_len_host, ho + B * L, B * 4);
     memcpy(match_len_host, ho + B * L + B, 2 * B * 4);

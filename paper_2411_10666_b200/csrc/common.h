@@ -24,7 +24,8 @@ struct sam_batch {
     size_t workspace_bytes;
     int32_t max_host_stride;
     size_t stage_words;           // int32 words of device staging
-    int32_t* host_stage;          // pinned host mirror of the staging area
+    int32_t* host_stage;          // pinned, device-mapped host staging area
+    int32_t* host_stage_dev;      // the same memory as the device addresses it
 };
 
 void sam_set_cuda_error(cudaError_t e);

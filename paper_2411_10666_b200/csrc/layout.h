@@ -50,7 +50,9 @@
 enum {
     CB_STATUS = 0, CB_NTOK, CB_NSTATES, CB_LAST, CB_S1, CB_L1, CB_S2, CB_L2,
     CB_S1FLAG, CB_BLK_CUR, CB_BLK_END, CB_NRECSLABS, CB_ROOTDEG, CB_RSV13, CB_RSV14, CB_RSV15,
-    CB_SLABTAB = 16   // .. 47
+    CB_SLABTAB = 16,  // .. 47
+    CB_REC1 = 48,     // .. 55: copy of the static match state's record (valid when s1 != 0)
+    CB_REC2 = 56      // .. 63: copy of the dynamic match state's record (valid when s2 != 0)
 };
 
 struct SamStaticRec {   // 32 bytes

@@ -54,11 +54,16 @@ __device__ __forceinline__ void gather_draft(const int32_t* text, int64_t e, int
     }
 }
 
+__device__ __forceinline__ void prefetch_l1(const void* p) {
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(__cvta_generic_to_global(p)));
+}
+
 // ------------------------------------------------------------------ static side
 // Transfer (Algorithm 1) for one token.  (s, sf, l): state, its F bit, match length.
-// root_e is root_row[t], fetched beforehand.
+// root_e is root_row[t], fetched beforehand.  If have_rec, (pa, pb) is the record of s, read earlier.
 __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t& s, uint32_t& sf, int32_t& l,
-                                                uint32_t t, uint32_t root_e, int lane, int& err) {
+                                                uint32_t t, uint32_t root_e, int lane, int& err,
+                                                bool have_rec, uint4 pa, uint4 pb) {
     int guard = l + 2;                       // at most l link moves
     bool len_from_rec = false;
     for (;;) {
@@ -70,8 +75,9 @@ __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t
         uint32_t home = sam_hash2(s, t) & S.hash_mask;
         uint4 ent = make_uint4(SAM_NONE, 0, 0, 0);
         if (sf) ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
-        const uint4 a = __ldg(S.rec + 2 * (size_t)s);
-        const uint4 b = __ldg(S.rec + 2 * (size_t)s + 1);
+        uint4 a = pa, b = pb;
+        if (!have_rec) { a = __ldg(S.rec + 2 * (size_t)s); b = __ldg(S.rec + 2 * (size_t)s + 1); }
+        have_rec = false;
         if (len_from_rec) { l = (int32_t)a.x; len_from_rec = false; }
         uint32_t tgt = SAM_NONE;
         if (a.w >= 1 && b.x == t) tgt = b.y;
@@ -159,9 +165,11 @@ __device__ __forceinline__ uint32_t alloc_block(Dyn& D, uint32_t cap) {
     return off;
 }
 
-__device__ __forceinline__ Look lookup_state(const Dyn& D, uint32_t p, uint32_t t) {
-    const uint4* rp = rec_ptr(D, p);
-    const uint4 a = rp[0], b = rp[1];
+__device__ __forceinline__ Look lookup_state(const Dyn& D, uint32_t p, uint32_t t,
+                                             bool have_rec = false, uint4 pa = make_uint4(0, 0, 0, 0),
+                                             uint4 pb = make_uint4(0, 0, 0, 0)) {
+    uint4 a = pa, b = pb;
+    if (!have_rec) { const uint4* rp = rec_ptr(D, p); a = rp[0]; b = rp[1]; }
     Look r;
     r.len = a.x; r.link = a.y; r.deg = a.w; r.b0 = b.x; r.b1 = b.y; r.b2 = b.z; r.b3 = b.w;
     r.found = false; r.tgt = 0; r.idx = 0;
@@ -246,8 +254,9 @@ __device__ __forceinline__ RootLook root_lookup(Dyn& D, uint32_t t) {
 
 // Expand (Algorithm 3) for token t, fused with the dynamic matcher's Transfer.
 // last: state of the whole text; ntok: text length; (s2, l2): match state = link[last], its length.
+// If have_rec, (pa, pb) is the record of s2 as it stands (read at the end of the previous step).
 __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, uint32_t& ntok,
-                                           uint32_t& s2, uint32_t& l2) {
+                                           uint32_t& s2, uint32_t& l2, bool have_rec, uint4 pa, uint4 pb) {
     const uint32_t k = ntok + 1;                       // max_length after this token
     const uint32_t c = D.n_states;
     ensure_rec(D, c);
@@ -286,7 +295,8 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             }
             break;
         }
-        lk = lookup_state(D, p, t);
+        lk = lookup_state(D, p, t, have_rec, pa, pb);
+        have_rec = false;
         if (lk.found) { found = true; qt = lk.tgt; plen = lk.len; break; }
         insert_edge(D, p, lk, t, c);                   // len[p] + 1 < k: not solid
         if (D.err) return;
@@ -372,12 +382,18 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __shared__ int32_t sh_l[2], sh_s[2], sh_dl[2], sh_err[2];
 
+    // Everything the step needs to get going is read in one round trip: the slot's 64 control
+    // words (state, slab table, copies of the two match states' records), its count, and the
+    // first 32 tokens of its row (read before the count is known; unused lanes are ignored).
     uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
     const uint32_t cw = cb[lane];                       // control words 0..31
+    const uint32_t cw2 = cb[32 + lane];                 // control words 32..63
+    const int m = A.counts[b];
+    int32_t tok_first = 0;
+    if (lane < A.stride) tok_first = toks[lane];
     int status = (int)__shfl_sync(FULL, cw, CB_STATUS);
     const uint32_t ntok0 = __shfl_sync(FULL, cw, CB_NTOK);
-    const int m = A.counts[b];
-    const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
     const int L = A.L;
     __syncthreads();          // both warps hold the slot's state as it was before either writes any of it
 
@@ -391,7 +407,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
             bool bad = false;
             for (int base = 0; base < m; base += 32) {
                 int i = base + lane;
-                if (i < m) { int t = toks[i]; bad |= (t < 0 || t >= vocab); }
+                if (i < m) { int t = base == 0 ? tok_first : toks[i]; bad |= (t < 0 || t >= vocab); }
             }
             if (__any_sync(FULL, bad)) status = SAM_SEQ_BAD_TOKEN;
         }
@@ -410,6 +426,14 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         return;
     }
 
+    // this warp's copy of its match state's record: words CB_REC1.. (warp 0) or CB_REC2.. (warp 1)
+    const int rbase = (warp == 0 ? CB_REC1 : CB_REC2) - 32;
+    uint4 ra, rb;
+    ra.x = __shfl_sync(FULL, cw2, rbase + 0); ra.y = __shfl_sync(FULL, cw2, rbase + 1);
+    ra.z = __shfl_sync(FULL, cw2, rbase + 2); ra.w = __shfl_sync(FULL, cw2, rbase + 3);
+    rb.x = __shfl_sync(FULL, cw2, rbase + 4); rb.y = __shfl_sync(FULL, cw2, rbase + 5);
+    rb.z = __shfl_sync(FULL, cw2, rbase + 6); rb.w = __shfl_sync(FULL, cw2, rbase + 7);
+
     int32_t d[MAX_DRAFT_REGS] = {-1, -1, -1, -1};
     int32_t my_l = 0, my_s = 0, my_dl = 0;
     int err = 0;
@@ -419,21 +443,32 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         if (A.has_static) {
             uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
             int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
+            bool have = s != 0;
             for (int base = 0; base < m && !err; base += 32) {
                 const int i = base + lane;
                 uint32_t tk = 0, re = SAM_NONE;
-                if (i < m) { tk = (uint32_t)toks[i]; re = __ldg(A.S.root_row + tk); }
+                if (i < m) { tk = (uint32_t)(base == 0 ? tok_first : toks[i]); re = __ldg(A.S.root_row + tk); }
                 const int cnt = min(32, m - base);
-                for (int j = 0; j < cnt && !err; j++)
-                    static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err);
+                for (int j = 0; j < cnt && !err; j++) {
+                    static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err,
+                                    have, ra, rb);
+                    have = false;
+                }
             }
-            if (m > 0 && lane == 0 && !err) { cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf; }
             my_l = l; my_s = (int32_t)s;
             if (l > 0 && !err) {
-                const int64_t e = (int64_t)__ldg(A.S.rec + 2 * (size_t)s).z;       // min_endpos
+                if (m > 0) {                                    // the state moved: read its record, keep a copy
+                    ra = __ldg(A.S.rec + 2 * (size_t)s);
+                    rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
+                }
+                const int64_t e = (int64_t)ra.z;                // min_endpos
                 int64_t room = A.S.n_tokens - e;
                 my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
                 gather_draft<true>(A.S.corpus, e, my_dl, L, lane, d);
+            }
+            if (m > 0 && lane == 0 && !err) {
+                cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf;
+                if (l > 0) { reinterpret_cast<uint4*>(cb + CB_REC1)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC1)[1] = rb; }
             }
         }
     } else {
@@ -444,7 +479,10 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         D.text = A.W.text + (size_t)b * A.W.text_stride;
         D.pool_hdr = A.W.pool_hdr; D.free_stack = A.W.free_stack; D.slab_owner = A.W.slab_owner;
         D.cb = cb;
-        D.tab = cb[CB_SLABTAB + lane];
+        {   // slab table entry i is control word 16 + i
+            uint32_t lo = __shfl_sync(FULL, cw, (lane + 16) & 31), hi = __shfl_sync(FULL, cw2, (lane + 16) & 31);
+            D.tab = lane < 16 ? lo : hi;
+        }
         D.n_rec_slabs = __shfl_sync(FULL, cw, CB_NRECSLABS);
         D.n_states = __shfl_sync(FULL, cw, CB_NSTATES);
         D.blk_cur = __shfl_sync(FULL, cw, CB_BLK_CUR);
@@ -457,15 +495,24 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         uint32_t s2 = __shfl_sync(FULL, cw, CB_S2), l2 = __shfl_sync(FULL, cw, CB_L2);
         if (D.n_states == 0) D.n_states = 1;            // the root exists implicitly (no record is read for it)
 
+        bool have = s2 != 0;
         for (int base = 0; base < m && !D.err; base += 32) {
             const int i = base + lane;
             uint32_t tk = 0;
-            if (i < m) tk = (uint32_t)toks[i];
+            if (i < m) {
+                tk = (uint32_t)(base == 0 ? tok_first : toks[i]);
+                // most walks end in the root table: bring each token's bucket (two lines) close now
+                const uint2* bk = D.root + (size_t)(sam_hash1(tk) & D.root_bmask) * SAM_ROOT_BUCKET;
+                prefetch_l1(bk); prefetch_l1(bk + 16);
+            }
             const int cnt = min(32, m - base);
-            for (int j = 0; j < cnt && !D.err; j++)
-                dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2);
+            for (int j = 0; j < cnt && !D.err; j++) {
+                dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2, have, ra, rb);
+                have = false;
+            }
         }
         err = D.err;
+        my_l = (int32_t)l2; my_s = (int32_t)s2;
         if (m > 0 && !err) {
             // the newest state's record, without a transition yet
             uint4* rl = rec_ptr(D, last);
@@ -478,9 +525,13 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
             }
             __syncwarp();
         }
-        my_l = (int32_t)l2; my_s = (int32_t)s2;
         if (l2 > 0 && !err) {
-            const int64_t e = (int64_t)rec_ptr(D, s2)[0].z;                       // min_endpos
+            if (m > 0) {                                        // the state moved: read its record, keep a copy
+                const uint4* rs = rec_ptr(D, s2);
+                ra = rs[0]; rb = rs[1];
+                if (lane == 0) { reinterpret_cast<uint4*>(cb + CB_REC2)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC2)[1] = rb; }
+            }
+            const int64_t e = (int64_t)ra.z;                    // min_endpos
             int64_t room = (int64_t)ntok - e;
             my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
             gather_draft<false>(D.text, e, my_dl, L, lane, d);
