@@ -43,6 +43,11 @@ UNIT = "sequence-steps/s"
 # and the input and output rows.
 ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.1}
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of sam_step_kernel from the committed ncu
+# capture (profiles/ncu_full_sam_step_kernel_c2.md); None for workloads without a capture of the
+# kernel as it stands.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 178261}
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -305,7 +310,7 @@ def main_ours(args):
     except Exception:
         peak = 6650.0
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_src + " stream copy",
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(base.name), "peak_source": peak_src + " stream copy",
                 "kernel": "sam_step_kernel", "launch_us": launch_us,
                 "algorithmic_bytes_per_sequence_step": algo_b,
                 "sequence_steps_per_launch": units / K}
