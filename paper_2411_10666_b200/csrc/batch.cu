@@ -39,7 +39,7 @@ int plan(const sam_batch_opts_t* o, WsLayout* w) {
     w->text_stride = (int32_t)sam_align_up((size_t)n, 32);
     // the root has at most one transition per text position: twice that many slots
     uint32_t rc = pow2_ceil((uint64_t)2 * n);
-    w->root_cap = rc < 2 * SAM_ROOT_BUCKET ? 2 * SAM_ROOT_BUCKET : (int32_t)rc;
+    w->root_cap = rc < 64 ? 64 : (int32_t)rc;             // never fewer than two 32-entry probe windows
     w->max_host_stride = o->max_host_stride ? o->max_host_stride : 32;
     w->stage_words = (size_t)o->batch * ((size_t)w->max_host_stride + 1 + (size_t)o->max_draft_len + 7);
 

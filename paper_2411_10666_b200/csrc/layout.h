@@ -23,8 +23,10 @@
 //               change once a state exists, so the bit is fixed when the transition is written and
 //               Expand's "p.length + 1 = q.length" test needs no read of q.
 //   block     : capacity (16 * 2^k) x 8-byte { tok, tgt | S }, first `deg` used, unordered.
-//   root table: per slot, buckets of 32 x 8-byte { tok, tgt | S } (256 bytes), open addressing
-//               by bucket; tok == SAM_NONE is empty.
+//   root table: per slot, 8-byte { tok, tgt | S } entries, linear probing from the start of the
+//               token's home bucket (8 entries = 64 bytes); tok == SAM_NONE is empty.  A warp reads
+//               32 consecutive entries per probe; a single lane can settle most lookups from the
+//               home bucket alone (found, or absent because the bucket still has an empty entry).
 //   text      : per slot, int32[max_seq_len].
 #pragma once
 #include <stdint.h>
@@ -41,7 +43,7 @@
 #define SAM_IDMASK 0x7FFFFFFFu
 
 #define SAM_HASH_BUCKET 8          // entries per static hash bucket (8 x 16 B = 128 B)
-#define SAM_ROOT_BUCKET 32         // entries per dynamic root-table bucket (32 x 8 B = 256 B)
+#define SAM_ROOT_BUCKET 8          // entries per dynamic root-table bucket (8 x 8 B = 64 B)
 #define SAM_BLOCK_MIN 16           // smallest dynamic edge block (16 x 8 B = 128 B)
 #define SAM_MAX_REC_SLABS 32       // entries of a slot's state-slab table (one per lane)
 #define SAM_CTRL_WORDS 64          // per-slot control block, 256 bytes

@@ -54,10 +54,6 @@ __device__ __forceinline__ void gather_draft(const int32_t* text, int64_t e, int
     }
 }
 
-__device__ __forceinline__ void prefetch_l1(const void* p) {
-    asm volatile("prefetch.global.L1 [%0];" ::"l"(__cvta_generic_to_global(p)));
-}
-
 // ------------------------------------------------------------------ static side
 // Transfer (Algorithm 1) for one token.  (s, sf, l): state, its F bit, match length.
 // root_e is root_row[t], fetched beforehand.  If have_rec, (pa, pb) is the record of s, read earlier.
@@ -110,6 +106,10 @@ struct Dyn {
     uint32_t tab;                // lane i: slab index of state slab i
     uint32_t n_rec_slabs, n_states, blk_cur, blk_end, root_deg, root_bmask;
     int slab_shift, rps_shift, seq, lane, err;
+    // Root-table lookups settled ahead of time, one lane per token of the current chunk of 32
+    // (root_precompute): pr_state 0 = not known (or stale), 1 = present, 2 = absent.
+    uint32_t pr_state, pr_tgt, pr_slot, pr_bucket;
+    int cur;                     // lane that holds the answer for the token being processed
 };
 
 struct Look {                    // result of looking a token up in a non-root state
@@ -233,30 +233,80 @@ __device__ __forceinline__ void insert_edge(Dyn& D, uint32_t p, const Look& lk, 
 
 struct RootLook { uint32_t tgt, slot; bool found; };
 
+// Each lane looks its own token up in the root table by itself: the home bucket (64 bytes, four
+// 16-byte reads) settles it when the token is there, or when the bucket still has an empty entry
+// (linear probing never skips one).  All tokens of the chunk are looked up in one round trip,
+// before any of them is processed; later changes to the table mark the affected answers stale.
+__device__ __forceinline__ void root_precompute(Dyn& D, uint32_t tk, bool valid) {
+    D.pr_state = 0; D.pr_tgt = 0; D.pr_slot = 0; D.pr_bucket = SAM_NONE;
+    if (!valid) return;
+    const uint32_t home = sam_hash1(tk) & D.root_bmask;
+    const uint4* bk = reinterpret_cast<const uint4*>(D.root + (size_t)home * SAM_ROOT_BUCKET);
+    uint4 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) v[i] = bk[i];
+    D.pr_bucket = home;
+    int first_empty = -1;
+#pragma unroll
+    for (int i = 3; i >= 0; i--) {                       // descending, so the lowest index wins
+        if (v[i].z == SAM_NONE) first_empty = 2 * i + 1;
+        if (v[i].x == SAM_NONE) first_empty = 2 * i;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        if (v[i].x == tk) { D.pr_state = 1; D.pr_tgt = v[i].y; D.pr_slot = home * SAM_ROOT_BUCKET + 2 * i; }
+        if (v[i].z == tk) { D.pr_state = 1; D.pr_tgt = v[i].w; D.pr_slot = home * SAM_ROOT_BUCKET + 2 * i + 1; }
+    }
+    if (D.pr_state == 0 && first_empty >= 0) { D.pr_state = 2; D.pr_slot = home * SAM_ROOT_BUCKET + first_empty; }
+}
+
 __device__ __forceinline__ RootLook root_lookup(Dyn& D, uint32_t t) {
     RootLook r; r.found = false; r.tgt = 0; r.slot = 0;
-    uint32_t bk = sam_hash1(t) & D.root_bmask;
-    for (uint32_t probe = 0; probe <= D.root_bmask; probe++) {
-        uint2 e = D.root[(size_t)bk * SAM_ROOT_BUCKET + D.lane];
+    const uint32_t st = __shfl_sync(FULL, D.pr_state, D.cur);
+    if (st != 0) {                                       // settled ahead of time and still current
+        r.found = st == 1;
+        r.tgt = __shfl_sync(FULL, D.pr_tgt, D.cur);
+        r.slot = __shfl_sync(FULL, D.pr_slot, D.cur);
+        return r;
+    }
+    const uint32_t cap_mask = (D.root_bmask + 1) * SAM_ROOT_BUCKET - 1;
+    const uint32_t base = (sam_hash1(t) & D.root_bmask) * SAM_ROOT_BUCKET;
+    for (uint32_t off = 0; off <= cap_mask; off += 32) {
+        uint2 e = D.root[(base + off + D.lane) & cap_mask];
         unsigned hit = __ballot_sync(FULL, e.x == t);
         if (hit) {
             int src = __ffs(hit) - 1;
-            r.found = true; r.tgt = __shfl_sync(FULL, e.y, src); r.slot = bk * SAM_ROOT_BUCKET + src;
+            r.found = true; r.tgt = __shfl_sync(FULL, e.y, src); r.slot = (base + off + src) & cap_mask;
             return r;
         }
         unsigned empty = __ballot_sync(FULL, e.x == SAM_NONE);
-        if (empty) { r.slot = bk * SAM_ROOT_BUCKET + (__ffs(empty) - 1); return r; }
-        bk = (bk + 1) & D.root_bmask;
+        if (empty) { r.slot = (base + off + (__ffs(empty) - 1)) & cap_mask; return r; }
     }
     D.err = SAM_SEQ_WALK_LIMIT;           // table full: cannot happen with root_cap >= 2 * distinct tokens
     return r;
 }
 
+// new root transition; answers settled ahead of time for the bucket it lands in are no longer current
+__device__ __forceinline__ void root_insert(Dyn& D, uint32_t slot, uint32_t t, uint32_t tgt) {
+    if (D.lane == 0) D.root[slot] = make_uint2(t, tgt);
+    if (D.pr_bucket == slot / SAM_ROOT_BUCKET) D.pr_state = 0;
+    __syncwarp();
+    D.root_deg++;
+}
+// change the target of an existing root transition
+__device__ __forceinline__ void root_retarget(Dyn& D, uint32_t slot, uint32_t tgt) {
+    if (D.lane == 0) D.root[slot].y = tgt;
+    if (D.pr_state == 1 && D.pr_slot == slot) D.pr_tgt = tgt;
+}
+
 // Expand (Algorithm 3) for token t, fused with the dynamic matcher's Transfer.
 // last: state of the whole text; ntok: text length; (s2, l2): match state = link[last], its length.
-// If have_rec, (pa, pb) is the record of s2 as it stands (read at the end of the previous step).
+// On entry, if have_rec, (pa, pb) is the record of s2 as it stands; on exit have_rec says whether
+// (pa, pb) is the record of the new s2 (known without a read when s2 is a fresh clone).
 __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, uint32_t& ntok,
-                                           uint32_t& s2, uint32_t& l2, bool have_rec, uint4 pa, uint4 pb) {
+                                           uint32_t& s2, uint32_t& l2, bool& have_rec, uint4& pa, uint4& pb) {
+    bool use_rec = have_rec;
+    have_rec = false;
     const uint32_t k = ntok + 1;                       // max_length after this token
     const uint32_t c = D.n_states;
     ensure_rec(D, c);
@@ -289,14 +339,12 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             if (D.err) return;
             if (rl.found) { found = true; at_root = true; qt = rl.tgt; plen = 0; root_slot = rl.slot; }
             else {
-                if (D.lane == 0) D.root[rl.slot] = make_uint2(t, c | (k == 1 ? SAM_FLAG : 0u));
-                __syncwarp();
-                D.root_deg++;
+                root_insert(D, rl.slot, t, c | (k == 1 ? SAM_FLAG : 0u));
             }
             break;
         }
-        lk = lookup_state(D, p, t, have_rec, pa, pb);
-        have_rec = false;
+        lk = lookup_state(D, p, t, use_rec, pa, pb);
+        use_rec = false;
         if (lk.found) { found = true; qt = lk.tgt; plen = lk.len; break; }
         insert_edge(D, p, lk, t, c);                   // len[p] + 1 < k: not solid
         if (D.err) return;
@@ -337,7 +385,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             __syncwarp();
             // redirect p and the states above it whose t-transition is q
             if (at_root) {
-                if (D.lane == 0) D.root[root_slot].y = cl | SAM_FLAG;
+                root_retarget(D, root_slot, cl | SAM_FLAG);
             } else {
                 uint32_t* rw = reinterpret_cast<uint32_t*>(rec_ptr(D, p));
                 if (D.lane == 0) {
@@ -350,9 +398,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
                     if (pp == 0) {
                         RootLook r2 = root_lookup(D, t);
                         if (D.err) return;
-                        if (r2.found && (r2.tgt & SAM_IDMASK) == q) {
-                            if (D.lane == 0) D.root[r2.slot].y = cl;
-                        }
+                        if (r2.found && (r2.tgt & SAM_IDMASK) == q) root_retarget(D, r2.slot, cl);
                         break;
                     }
                     Look l2k = lookup_state(D, pp, t);
@@ -370,10 +416,53 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             if (D.lane == 0) reinterpret_cast<uint32_t*>(rq)[1] = cl;        // link[q] = cl
             __syncwarp();
             s2 = cl; l2 = plen + 1;
+            have_rec = true;                                                 // cl's record as just written
+            pa = make_uint4(plen + 1, qa.y, qa.z, qa.w); pb = nb;
         }
     }
     if (D.lane == 0) D.text[ntok] = (int32_t)t;
     last = c; ntok = k;
+}
+
+// A run of tokens that are all new to the sequence, met while nothing is matched (s2 is the root):
+// Expand for each of them is the same three writes — the previous state's record with its one
+// solid transition, a root transition, the text — and none depends on another, so lanes j..j+r-1
+// do one token each at once.  A token qualifies if its root lookup was settled ahead of time as
+// "absent" and no earlier token of the run shares its home bucket (so slots and tokens differ).
+// Returns r (0 if token j does not qualify).
+__device__ __forceinline__ int dyn_fresh_run(Dyn& D, uint32_t tk, int j, int cnt, unsigned bucket_peers,
+                                             uint32_t& last, uint32_t& ntok) {
+    const unsigned from_j = ~((1u << j) - 1u);
+    const unsigned lt = (1u << D.lane) - 1u;
+    const bool first_of_bucket = (bucket_peers & from_j & lt) == 0;
+    const unsigned elig = __ballot_sync(FULL, D.pr_state == 2 && first_of_bucket && D.lane >= j && D.lane < cnt);
+    const unsigned gap = ~(elig >> j);
+    int r = gap ? __ffs(gap) - 1 : 32 - j;
+    if (r <= 0) return 0;
+    const uint32_t c0 = D.n_states;
+    ensure_rec(D, c0);
+    if (!D.err) ensure_rec(D, c0 + r - 1);
+    if (D.err) return 0;
+    const int idx = D.lane - j;
+    const bool mine = idx >= 0 && idx < r;
+    const uint32_t c = c0 + (uint32_t)idx;
+    const uint32_t prev = idx == 0 ? last : c - 1;            // the state this token's transition leaves
+    const uint32_t plen = ntok + (uint32_t)idx;               // its length = tokens before this one
+    uint4* rp = rec_ptr(D, mine ? prev : 1u);
+    if (mine) {
+        if (prev != 0) {
+            rp[0] = make_uint4(plen, 0, plen, 1);             // link is the root: nothing was matched
+            rp[1] = make_uint4(tk, c | SAM_FLAG, 0, 0);
+        }
+        D.root[D.pr_slot] = make_uint2(tk, c | (plen == 0 ? SAM_FLAG : 0u));
+        D.text[plen] = (int32_t)tk;
+    }
+    const unsigned run = ((r >= 32 ? 0u : (1u << r)) - 1u) << j;
+    if (bucket_peers & run) D.pr_state = 0;                   // those buckets changed
+    __syncwarp();
+    D.n_states = c0 + r; D.root_deg += r;
+    last = c0 + r - 1; ntok += r;
+    return r;
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -491,6 +580,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         D.root_bmask = (uint32_t)(A.W.root_cap / SAM_ROOT_BUCKET) - 1;
         D.slab_shift = A.W.slab_shift; D.rps_shift = A.W.slab_shift - 5;
         D.seq = b; D.lane = lane; D.err = 0;
+        D.pr_state = 0; D.pr_tgt = 0; D.pr_slot = 0; D.pr_bucket = SAM_NONE; D.cur = 0;
         uint32_t last = __shfl_sync(FULL, cw, CB_LAST), ntok = ntok0;
         uint32_t s2 = __shfl_sync(FULL, cw, CB_S2), l2 = __shfl_sync(FULL, cw, CB_L2);
         if (D.n_states == 0) D.n_states = 1;            // the root exists implicitly (no record is read for it)
@@ -499,16 +589,20 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         for (int base = 0; base < m && !D.err; base += 32) {
             const int i = base + lane;
             uint32_t tk = 0;
-            if (i < m) {
-                tk = (uint32_t)(base == 0 ? tok_first : toks[i]);
-                // most walks end in the root table: bring each token's bucket (two lines) close now
-                const uint2* bk = D.root + (size_t)(sam_hash1(tk) & D.root_bmask) * SAM_ROOT_BUCKET;
-                prefetch_l1(bk); prefetch_l1(bk + 16);
-            }
+            if (i < m) tk = (uint32_t)(base == 0 ? tok_first : toks[i]);
+            root_precompute(D, tk, i < m);              // most walks end in the root table
+            const unsigned bucket_peers = __match_any_sync(FULL, D.pr_bucket);
             const int cnt = min(32, m - base);
-            for (int j = 0; j < cnt && !D.err; j++) {
+            int j = 0;
+            while (j < cnt && !D.err) {
+                if (s2 == 0) {
+                    const int r = dyn_fresh_run(D, tk, j, cnt, bucket_peers, last, ntok);
+                    if (r > 0) { j += r; have = false; continue; }
+                    if (D.err) break;
+                }
+                D.cur = j;
                 dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2, have, ra, rb);
-                have = false;
+                j++;
             }
         }
         err = D.err;
@@ -526,9 +620,8 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
             __syncwarp();
         }
         if (l2 > 0 && !err) {
-            if (m > 0) {                                        // the state moved: read its record, keep a copy
-                const uint4* rs = rec_ptr(D, s2);
-                ra = rs[0]; rb = rs[1];
+            if (m > 0) {                                        // the state moved: get its record, keep a copy
+                if (!have) { const uint4* rs = rec_ptr(D, s2); ra = rs[0]; rb = rs[1]; }
                 if (lane == 0) { reinterpret_cast<uint4*>(cb + CB_REC2)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC2)[1] = rb; }
             }
             const int64_t e = (int64_t)ra.z;                    // min_endpos
