@@ -54,7 +54,7 @@ enum {
 };
 
 /* source_dev values */
-enum { SAM_SRC_NONE = 0, SAM_SRC_STATIC = 1, SAM_SRC_DYNAMIC = 2 };
+enum { SAM_SRC_NONE = 0, SAM_SRC_STATIC = 1, SAM_SRC_DYNAMIC = 2, SAM_SRC_AUXILIARY = 3 };
 
 typedef struct sam_static sam_static_t;   /* device-resident static automaton, owned by the library */
 typedef struct sam_batch sam_batch_t;     /* batch of sequences; its device memory is the caller's  */
@@ -214,6 +214,35 @@ int sam_batch_pool_info(sam_batch_t* b, int64_t* total_slabs, int64_t* free_slab
 
 /* Forget the batch.  The workspace is the caller's and is not freed. */
 void sam_batch_destroy(sam_batch_t* b);
+
+/* ---- closing the loop on the device -------------------------------------------------------- */
+
+/* Greedy verification (Section 2.2): the target model has scored the draft; target_tokens_dev[i, j]
+ * is its token for the position after the first j draft tokens (j = 0..L, so row i has L + 1
+ * entries, of which draft_len[i] + 1 are read).  Slot i accepts a = the length of the longest
+ * prefix of its draft that equals target[i, 0..a), and its accepted tokens x_accept are
+ * target[i, 0..a] — the a confirmed draft tokens and the target's own next token — so
+ * m = a + 1, clipped to `stride` and, if max_new_dev is given, to max_new_dev[i] (0 stops a slot).
+ * Writes counts_dev[i] = m and new_tokens_dev[i, 0..m) (-1 beyond), ready to be the next sam_step's
+ * input, and accepted_dev[i] = min(a, m) if accepted_dev is not NULL.
+ *   draft_tokens_dev device int32 [B, L]; draft_len_dev [B]; target_tokens_dev [B, L+1];
+ *   max_new_dev [B] or NULL; new_tokens_dev [B, stride]; counts_dev [B]; accepted_dev [B] or NULL.
+ * Asynchronous on `stream`.  Errors: ARG, CUDA. */
+int sam_accept_greedy(int32_t batch, const int32_t* draft_tokens_dev, const int32_t* draft_len_dev, int32_t L,
+                      const int32_t* target_tokens_dev, const int32_t* max_new_dev,
+                      int32_t* new_tokens_dev, int32_t stride, int32_t* counts_dev, int32_t* accepted_dev,
+                      void* stream);
+
+/* Adaptive draft selection (Section 3.4): the auxiliary drafter stands in with a fixed virtual match
+ * length l_threshold.  With min_match = l_threshold in sam_batch_opts_t, sam_step reports
+ * source = SAM_SRC_NONE exactly where the automaton's chosen match is shorter than that; this call
+ * then substitutes the auxiliary draft there, in place: for every slot with source == SAM_SRC_NONE
+ * and aux_len > 0, draft_tokens[i, :] = aux_tokens[i, 0..aux_len) (-1 beyond), draft_len = aux_len,
+ * source = SAM_SRC_AUXILIARY.  aux_tokens_dev device int32 [B, L]; aux_len_dev [B].
+ * Asynchronous on `stream`.  Errors: ARG, CUDA. */
+int sam_select_auxiliary(int32_t batch, int32_t L, int32_t* draft_tokens_dev, int32_t* draft_len_dev,
+                         int32_t* source_dev, const int32_t* aux_tokens_dev, const int32_t* aux_len_dev,
+                         void* stream);
 
 /* ---- retrieval without any allocation ------------------------------------------------------ */
 

@@ -18,7 +18,7 @@ _lib = None
 SAM_OK = 0
 ERR_NAMES = {-1: "ARG", -2: "CUDA", -3: "NOMEM", -4: "WORKSPACE", -5: "IO", -6: "FORMAT", -7: "LIMIT", -8: "NO_DEVICE"}
 SEQ_OK, SEQ_CAPACITY, SEQ_WALK_LIMIT, SEQ_BAD_TOKEN, SEQ_BAD_COUNT = 0, 1, 2, 3, 4
-SRC_NONE, SRC_STATIC, SRC_DYNAMIC = 0, 1, 2
+SRC_NONE, SRC_STATIC, SRC_DYNAMIC, SRC_AUXILIARY = 0, 1, 2, 3
 
 
 class SamError(RuntimeError):
@@ -74,6 +74,9 @@ SIGNATURES = {
                                c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "sam_batch_pool_info": (c_int, [c_void_p, POINTER(c_int64), POINTER(c_int64), c_void_p]),
     "sam_batch_destroy": (None, [c_void_p]),
+    "sam_accept_greedy": (c_int, [c_int32, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32,
+                                  c_void_p, c_void_p, c_void_p]),
+    "sam_select_auxiliary": (c_int, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "sam_retrieve_noalloc": (c_int, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32,
                                      c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "sam_noalloc_capacity_bytes": (c_size_t, []),
@@ -270,6 +273,21 @@ def sam_batch_pool_info(h, stream=None):
     tot, free = c_int64(), c_int64()
     _check(lib().sam_batch_pool_info(h, byref(tot), byref(free), _stream_ptr(stream)), "sam_batch_pool_info")
     return tot.value, free.value
+
+
+def sam_accept_greedy(draft_tokens, draft_len, target_tokens, max_new, new_tokens, counts, accepted=None, stream=None):
+    B, L = draft_tokens.shape
+    _check(lib().sam_accept_greedy(B, _dev_ptr(draft_tokens, "draft_tokens"), _dev_ptr(draft_len, "draft_len"), L,
+                                   _dev_ptr(target_tokens, "target_tokens"), _dev_ptr(max_new, "max_new"),
+                                   _dev_ptr(new_tokens, "new_tokens"), new_tokens.shape[1], _dev_ptr(counts, "counts"),
+                                   _dev_ptr(accepted, "accepted"), _stream_ptr(stream)), "sam_accept_greedy")
+
+
+def sam_select_auxiliary(draft_tokens, draft_len, source, aux_tokens, aux_len, stream=None):
+    B, L = draft_tokens.shape
+    _check(lib().sam_select_auxiliary(B, L, _dev_ptr(draft_tokens, "draft_tokens"), _dev_ptr(draft_len, "draft_len"),
+                                      _dev_ptr(source, "source"), _dev_ptr(aux_tokens, "aux_tokens"),
+                                      _dev_ptr(aux_len, "aux_len"), _stream_ptr(stream)), "sam_select_auxiliary")
 
 
 def sam_retrieve_noalloc(static_h, vocab, tokens, counts, L, l_bias, min_match,

@@ -1,0 +1,89 @@
+"""GPU: greedy verification, auxiliary selection and the closed decoding loop against the oracle."""
+import random
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+from oracle import accept
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2411_10666_b200 as pkg
+    pkg.lib()
+    return pkg
+
+
+def _t(a, dev="cuda"):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(np.asarray(a, dtype=np.int32))).to(dev)
+
+
+def test_accept_and_select_random(P):
+    import torch
+    rng = np.random.default_rng(7)
+    for B, L, stride in [(1, 1, 1), (5, 4, 5), (37, 32, 33), (64, 40, 16), (300, 128, 129)]:
+        target = rng.integers(0, 4, size=(B, L + 1), dtype=np.int32)
+        draft = target[:, :L].copy()
+        flip = rng.random((B, L)) < 0.08
+        draft[flip] = (draft[flip] + 1) % 4
+        dlen = rng.integers(0, L + 1, size=B, dtype=np.int32)
+        cap = rng.integers(0, L + 3, size=B, dtype=np.int32)
+        for use_cap in (False, True):
+            nt, cnt, acc = accept.accept_greedy(draft, dlen, target, cap if use_cap else None, stride)
+            g_nt = torch.empty((B, stride), dtype=torch.int32, device="cuda")
+            g_cnt = torch.empty(B, dtype=torch.int32, device="cuda"); g_acc = torch.empty_like(g_cnt)
+            P.binding.sam_accept_greedy(_t(draft), _t(dlen), _t(target), _t(cap) if use_cap else None, g_nt, g_cnt, g_acc)
+            assert np.array_equal(g_nt.cpu().numpy(), nt) and np.array_equal(g_cnt.cpu().numpy(), cnt)
+            assert np.array_equal(g_acc.cpu().numpy(), acc)
+        src = rng.integers(0, 3, size=B, dtype=np.int32)
+        aux = rng.integers(0, 9, size=(B, L), dtype=np.int32); alen = rng.integers(0, L + 1, size=B, dtype=np.int32)
+        dd = np.where(np.arange(L)[None, :] < dlen[:, None], draft, -1).astype(np.int32)
+        e_d, e_l, e_s = accept.select_auxiliary(dd, dlen, src, aux, alen)
+        g_d, g_l, g_s = _t(dd), _t(dlen), _t(src)
+        P.binding.sam_select_auxiliary(g_d, g_l, g_s, _t(aux), _t(alen))
+        assert np.array_equal(g_d.cpu().numpy(), e_d) and np.array_equal(g_l.cpu().numpy(), e_l)
+        assert np.array_equal(g_s.cpu().numpy(), e_s)
+
+
+@pytest.mark.parametrize("key,N,B,pl,gl,min_match", [("tiny", 30000, 4, 64, 300, 1), ("c2", 300000, 16, 256, 400, 1),
+                                                      ("c4", 100000, 24, 600, 300, 3)])
+def test_closed_loop_matches_oracle(P, key, N, B, pl, gl, min_match):
+    """draft -> verify against the true continuation -> accept -> update, entirely on the device,
+    step for step equal to the same loop run by the oracle."""
+    import torch
+    spec = W.scaled(W.SPECS[key], N, B, pl, gl)
+    w = W.make(spec)
+    L, total, stride = spec.draft_len, pl + gl, spec.draft_len + 1
+    S = oracle.Sam(w.corpus)
+    ob = oracle.Batch(S, w.corpus, B, spec.vocab, total, 0, min_match)
+    log, pos_ref = accept.decode_loop(ob, w.seqs, pl, L, stride)
+
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    batch = P.Batch(st, B, total, max_draft_len=L, min_match=min_match)
+    dev = batch.device
+    seqs = _t(w.seqs, dev).long()
+    out = batch.step(_t(w.prompts, dev), torch.full((B,), pl, dtype=torch.int32, device=dev), L)
+    pos = torch.full((B,), pl, dtype=torch.int64, device=dev)
+    nt = torch.empty((B, stride), dtype=torch.int32, device=dev)
+    cnt = torch.empty(B, dtype=torch.int32, device=dev); acc = torch.empty_like(cnt)
+    ar = torch.arange(L + 1, device=dev)[None, :]
+    for step, ref in enumerate(log):
+        target = torch.gather(seqs, 1, torch.clamp(pos[:, None] + ar, max=total - 1)).int().contiguous()
+        cap = (total - pos).int().contiguous()
+        P.binding.sam_accept_greedy(out.draft_tokens, out.draft_len, target, cap, nt, cnt, acc)
+        got = out.cpu()
+        for k in ("draft_tokens", "draft_len", "match_len", "source", "state", "status"):
+            assert np.array_equal(got[k], ref[k]), (step, k)
+        assert np.array_equal(cnt.cpu().numpy(), ref["counts"]) and np.array_equal(acc.cpu().numpy(), ref["accepted"])
+        out = batch.step(nt, cnt, L, out)                     # no host round trip between verify and update
+        pos += cnt.long()
+    assert np.array_equal(pos.cpu().numpy(), pos_ref) and (pos_ref == total).all()
+    mean_accept = np.mean([r["counts"][r["counts"] > 0].mean() for r in log if (r["counts"] > 0).any()])
+    assert mean_accept > 1.05                                 # retrieval drafts do get accepted
