@@ -86,6 +86,9 @@ typedef struct {
     int32_t max_host_stride;  /* largest stride sam_step_host accepts; 0 = 32                  */
     int32_t slab_bytes;       /* slab size, a power of two >= 4 KiB; 0 = max(16 KiB, pow2 >= 8*max_seq_len) */
     int64_t pool_slabs;       /* slabs in the shared pool; 0 = batch * (ceil(160 * max_seq_len / slab_bytes) + 2) */
+    int32_t stop_token_plus_one; /* 0 = none; t + 1 = a draft ends before the first token t (e.g. the EOS
+                                  that separates the documents of a concatenated corpus, Section 3.1) */
+    int32_t reserved;         /* must be 0 */
 } sam_batch_opts_t;
 
 /* ---- static automaton -------------------------------------------------------------------- */

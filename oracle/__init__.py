@@ -60,7 +60,7 @@ def _load():
     lib.osam_tables.argtypes = [vp, _i32p, _i32p, _i32p, _i32p]
     lib.osam_counters.argtypes = [vp, _i64p]
     lib.obatch_new.restype = vp
-    lib.obatch_new.argtypes = [vp, _i32p, i64, i32, i32, i32, i32, i32]
+    lib.obatch_new.argtypes = [vp, _i32p, i64, i32, i32, i32, i32, i32, i32]
     lib.obatch_free.argtypes = [vp]
     lib.obatch_reset.argtypes = [vp, i32]
     lib.obatch_step.restype = ctypes.c_int
@@ -186,7 +186,7 @@ class Batch:
     """B decoding sequences over one shared static automaton (Sections 3.2, 3.3)."""
 
     def __init__(self, static: Sam | None, corpus, batch: int, vocab: int, max_seq_len: int,
-                 l_bias: int = 0, min_match: int = 1):
+                 l_bias: int = 0, min_match: int = 1, stop_token: int = -1):
         lib = _load()
         self._lib = lib
         self._static = static
@@ -195,7 +195,7 @@ class Batch:
         cp = _p32(self._corpus) if self._corpus is not None else ctypes.cast(None, _i32p)
         cn = 0 if self._corpus is None else self._corpus.shape[0]
         self._h = lib.obatch_new(static._h if static is not None else None, cp, cn,
-                                 batch, vocab, max_seq_len, l_bias, min_match)
+                                 batch, vocab, max_seq_len, l_bias, min_match, stop_token)
 
     def close(self):
         if self._h:

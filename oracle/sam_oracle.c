@@ -236,6 +236,8 @@ void osam_counters(const osam_t* S, int64_t* out) {
  *   - a chosen match shorter than max(1, min_match) yields no draft (source 0).
  *   - ties go to the dynamic automaton (strict >).
  *   - a draft is clipped at the end of the text; no wrap-around.
+ *   - with a stop token set (the EOS that joins the corpus' documents, Section 3.1) a draft ends
+ *     before its first occurrence.
  * Boundary conventions of the library that the oracle mirrors so whole arrays compare equal:
  *   status 1: n + m > max_seq_len; 3: a token outside [0, vocab); 4: m < 0 or m > stride.
  *   A sequence with a non-zero status is frozen from then on and reports zeros / -1 drafts.
@@ -245,6 +247,7 @@ typedef struct {
     const osam_t* st;           /* static automaton or NULL */
     const int32_t* corpus; int64_t corpus_len;
     int32_t batch, vocab, max_seq_len, l_bias, min_match;
+    int32_t stop_token;         /* a draft ends before the first such token; -1 = none */
     osam_t** dyn;               /* [batch] */
     int32_t** text;             /* [batch][max_seq_len] */
     int32_t *n, *s1, *l1, *s2, *l2, *status;
@@ -256,11 +259,11 @@ typedef struct {
 
 obatch_t* obatch_new(const osam_t* st, const int32_t* corpus, int64_t corpus_len,
                      int32_t batch, int32_t vocab, int32_t max_seq_len,
-                     int32_t l_bias, int32_t min_match) {
+                     int32_t l_bias, int32_t min_match, int32_t stop_token) {
     obatch_t* B = (obatch_t*)calloc(1, sizeof(obatch_t));
     B->st = st; B->corpus = corpus; B->corpus_len = corpus_len;
     B->batch = batch; B->vocab = vocab; B->max_seq_len = max_seq_len;
-    B->l_bias = l_bias; B->min_match = min_match;
+    B->l_bias = l_bias; B->min_match = min_match; B->stop_token = stop_token;
     B->dyn = (osam_t**)calloc((size_t)batch, sizeof(osam_t*));
     B->text = (int32_t**)calloc((size_t)batch, sizeof(int32_t*));
     B->n = (int32_t*)calloc((size_t)batch, 4); B->s1 = (int32_t*)calloc((size_t)batch, 4);
@@ -330,6 +333,8 @@ static void step_one(obatch_t* B, int32_t b, const int32_t* toks, int32_t stride
     int64_t n_text = use_static ? B->corpus_len : B->n[b];
     int64_t p = use_static ? B->st->min_endpos[B->s1[b]] : D->min_endpos[B->s2[b]];
     int64_t dl = n_text - p; if (dl > L) dl = L; if (dl < 0) dl = 0;             /* d = T[p+1 : p+n], clipped */
+    if (B->stop_token >= 0)                                                      /* stop at a document separator */
+        for (int64_t i = 0; i < dl; i++) if (text[p + i] == B->stop_token) { dl = i; break; }
     for (int64_t i = 0; i < dl; i++) draft[i] = text[p + i];
     *draft_len = (int32_t)dl;
     cnt[5] += dl;

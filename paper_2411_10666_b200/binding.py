@@ -44,7 +44,8 @@ class StaticInfo(Structure):
 class BatchOpts(Structure):
     _fields_ = [("batch", c_int32), ("max_seq_len", c_int32), ("max_draft_len", c_int32),
                 ("l_bias", c_int32), ("min_match", c_int32), ("vocab", c_int32),
-                ("max_host_stride", c_int32), ("slab_bytes", c_int32), ("pool_slabs", c_int64)]
+                ("max_host_stride", c_int32), ("slab_bytes", c_int32), ("pool_slabs", c_int64),
+                ("stop_token_plus_one", c_int32), ("reserved", c_int32)]
 
 
 _i32p = POINTER(c_int32)
@@ -379,7 +380,7 @@ class Batch:
 
     def __init__(self, static: StaticSam | None, batch: int, max_seq_len: int, max_draft_len: int = 32,
                  l_bias: int = 0, min_match: int = 1, vocab: int = 0, max_host_stride: int = 0,
-                 slab_bytes: int = 0, pool_slabs: int = 0, device: int | None = None):
+                 slab_bytes: int = 0, pool_slabs: int = 0, device: int | None = None, stop_token: int = -1):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("samdraft needs a CUDA device; there is no CPU path")
@@ -387,7 +388,7 @@ class Batch:
         dev = static.device if static is not None else (0 if device is None else device)
         self.device = torch.device("cuda", dev)
         self.opts = BatchOpts(batch, max_seq_len, max_draft_len, l_bias, min_match, vocab,
-                              max_host_stride, slab_bytes, pool_slabs)
+                              max_host_stride, slab_bytes, pool_slabs, stop_token + 1, 0)
         nbytes = sam_batch_workspace_bytes(self.opts)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)

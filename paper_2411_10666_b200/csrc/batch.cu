@@ -20,7 +20,8 @@ inline uint32_t pow2_ceil(uint64_t x) { uint64_t p = 1; while (p < x) p <<= 1; r
 
 int plan(const sam_batch_opts_t* o, WsLayout* w) {
     if (!o || o->batch < 1 || o->max_seq_len < 1 || o->max_draft_len < 1 || o->max_draft_len > 128 ||
-        o->l_bias < 0 || o->min_match < 0 || o->max_host_stride < 0 || o->pool_slabs < 0)
+        o->l_bias < 0 || o->min_match < 0 || o->max_host_stride < 0 || o->pool_slabs < 0 ||
+        o->stop_token_plus_one < 0 || o->reserved != 0)
         return SAM_ERR_ARG;
     if (o->max_seq_len > (1 << 28) || o->batch > (1 << 24)) return SAM_ERR_LIMIT;
     const int64_t n = o->max_seq_len;
@@ -178,6 +179,7 @@ int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBa
         view->l_bias = opts->l_bias; view->min_match = opts->min_match;
         view->vocab = vocab;
         view->pool_slabs = w.pool_slabs;
+        view->stop_token = opts->stop_token_plus_one - 1;
     }
     return SAM_OK;
 }
@@ -243,6 +245,7 @@ extern "C" int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* 
     V.l_bias = opts->l_bias; V.min_match = opts->min_match;
     V.vocab = st ? st->info.vocab : opts->vocab;
     V.pool_slabs = w.pool_slabs;
+    V.stop_token = opts->stop_token_plus_one - 1;
 
     SamDeviceGuard guard(b->device);
     if (!guard.ok) { delete b; return SAM_ERR_CUDA; }

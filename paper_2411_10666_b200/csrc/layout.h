@@ -108,4 +108,5 @@ struct SamBatchView {
     int32_t slab_shift;       // log2(slab_bytes)
     int32_t l_bias, min_match, vocab;
     int32_t pool_slabs;
+    int32_t stop_token;       // drafts end before the first such token; -1 = none
 };

@@ -64,6 +64,7 @@ extern "C" int sam_retrieve_noalloc(const sam_static_t* st, int32_t vocab, int32
     sam_batch_opts_t o;
     o.batch = batch; o.max_seq_len = stride; o.max_draft_len = L; o.l_bias = l_bias; o.min_match = min_match;
     o.vocab = st ? st->info.vocab : vocab; o.max_host_stride = 1; o.slab_bytes = 0; o.pool_slabs = 0;
+    o.stop_token_plus_one = 0; o.reserved = 0;
     size_t need = 0;
     int rc = sam_plan_view(&o, o.vocab, nullptr, nullptr, &need, nullptr);
     if (rc) return rc;

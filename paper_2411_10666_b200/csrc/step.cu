@@ -54,6 +54,20 @@ __device__ __forceinline__ void gather_draft(const int32_t* text, int64_t e, int
     }
 }
 
+// A draft ends before the first stop token (the separator between documents of a concatenated
+// corpus): returns the shortened length and blanks the lanes from there on.
+__device__ __forceinline__ int cut_at_stop(int32_t d[MAX_DRAFT_REGS], int dl, int lane, int32_t stop) {
+    if (stop < 0) return dl;
+#pragma unroll
+    for (int r = 0; r < MAX_DRAFT_REGS; r++) {
+        const unsigned hit = __ballot_sync(FULL, r * 32 + lane < dl && d[r] == stop);
+        if (hit) { dl = r * 32 + __ffs(hit) - 1; break; }
+    }
+#pragma unroll
+    for (int r = 0; r < MAX_DRAFT_REGS; r++) if (r * 32 + lane >= dl) d[r] = -1;
+    return dl;
+}
+
 // ------------------------------------------------------------------ static side
 // Transfer (Algorithm 1) for one token.  (s, sf, l): state, its F bit, match length.
 // root_e is root_row[t], fetched beforehand.  If have_rec, (pa, pb) is the record of s, read earlier.
@@ -554,6 +568,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                 int64_t room = A.S.n_tokens - e;
                 my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
                 gather_draft<true>(A.S.corpus, e, my_dl, L, lane, d);
+                my_dl = cut_at_stop(d, my_dl, lane, A.W.stop_token);
             }
             if (m > 0 && lane == 0 && !err) {
                 cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf;
@@ -628,6 +643,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
             int64_t room = (int64_t)ntok - e;
             my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
             gather_draft<false>(D.text, e, my_dl, L, lane, d);
+            my_dl = cut_at_stop(d, my_dl, lane, A.W.stop_token);
         }
     }
 

@@ -8,11 +8,11 @@ KEYS = ("draft_tokens", "draft_len", "match_len", "source", "state", "status")
 
 
 def oracle_run(corpus, vocab, prompts, new_tokens, counts, L, max_seq_len, l_bias=0, min_match=1,
-               static=None, threads=1):
+               static=None, threads=1, stop_token=-1):
     """Returns (per-step dict of arrays with a leading step axis incl. the prefill step, batch obj)."""
     B = prompts.shape[0]
     S = static if static is not None else (oracle.Sam(corpus) if corpus is not None else None)
-    ob = oracle.Batch(S, corpus, B, vocab, max_seq_len, l_bias, min_match)
+    ob = oracle.Batch(S, corpus, B, vocab, max_seq_len, l_bias, min_match, stop_token)
     outs = []
     if prompts.shape[1] > 0:
         outs.append(ob.step(prompts, np.full(B, prompts.shape[1], dtype=np.int32), L, threads))

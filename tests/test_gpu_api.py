@@ -195,3 +195,18 @@ def test_probes_report_plausible_numbers(P):
     ns1 = P.binding.sam_probe_chase(buf, 20000, chains=1)
     ns64 = P.binding.sam_probe_chase(buf, 20000, chains=64)
     assert 100 < ns1 < 5000 and 100 < ns64 < 5000
+
+
+def test_stop_token_matches_oracle(P):
+    spec = W.scaled(W.SPECS["tiny"], corpus_len=40_000, batch=6, prompt_len=100, gen_len=300)
+    w = W.make(spec)
+    L, msl = 40, spec.prompt_len + spec.gen_len
+    vals, cnts = np.unique(w.corpus, return_counts=True)
+    stop = int(vals[np.argmax(cnts)])                       # the most frequent token plays the separator
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, _, _ = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, stop_token=stop)
+    got, _ = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, stop_token=stop)
+    assert_same(got, ref)
+    plain, _ = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    assert (got["draft_len"] < plain["draft_len"]).any()    # some drafts were cut
+    assert not (got["draft_tokens"] == stop).any()

@@ -287,3 +287,26 @@ def test_workload_scale_self_certification():
                 assert (out.draft_tokens[b, :dl] == x[e2:e2 + dl]).all()
     assert n_static > 0
     assert B.counters()["tokens"] == spec.batch * (spec.prompt_len + spec.gen_len)
+
+
+def test_stop_token_cuts_the_draft_at_a_document_separator():
+    """Section 3.1 joins the corpus' documents with an EOS symbol; with that symbol as the stop token a
+    draft is the definition's draft cut before its first EOS."""
+    rng = random.Random(21)
+    EOS = 0
+    for _ in range(60):
+        docs = [[rng.randrange(1, 5) for _ in range(rng.randint(1, 9))] for _ in range(rng.randint(1, 8))]
+        corpus = [t for d in docs for t in d + [EOS]]
+        x = [rng.randrange(0, 5) for _ in range(rng.randint(1, 30))]
+        L = rng.randint(1, 8)
+        B = oracle.Batch(oracle.Sam(corpus), corpus, 1, 5, len(x), 0, 1, EOS)
+        for k in range(1, len(x) + 1):
+            out = B.step([[x[k - 1]]], [1], L)
+            exp = bf.retrieve(corpus, x, k, L)
+            d = exp["draft"]
+            if EOS in d:
+                d = d[:d.index(EOS)]
+            dl = int(out.draft_len[0])
+            assert out.source[0] == exp["source"]
+            assert out.draft_tokens[0, :dl].tolist() == d and (out.draft_tokens[0, dl:] == -1).all()
+            assert EOS not in out.draft_tokens[0, :dl].tolist()
