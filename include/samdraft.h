@@ -62,6 +62,8 @@ typedef struct sam_batch sam_batch_t;     /* batch of sequences; its device memo
 typedef struct {
     double hash_load;        /* target load of the overflow-edge hash table, (0, 0.9]; 0 = 0.5 */
     int32_t keep_host_copy;  /* reserved, must be 0                                            */
+    int32_t tree_topk;       /* 0 = no tree-draft data; k in 1..6 = also compute freq and the k most
+                                frequent successors of every state (Appendix A.2) for sam_tree_draft */
 } sam_build_opts_t;
 
 typedef struct {
@@ -74,6 +76,8 @@ typedef struct {
     int32_t vocab;
     size_t device_bytes;     /* device memory held                                             */
     double build_seconds;    /* host construction time (0 for a loaded image)                  */
+    int32_t tree_topk;       /* k the tree-draft data was built with (0: none)                 */
+    int32_t reserved;
 } sam_static_info_t;
 
 typedef struct {
@@ -246,6 +250,32 @@ int sam_accept_greedy(int32_t batch, const int32_t* draft_tokens_dev, const int3
 int sam_select_auxiliary(int32_t batch, int32_t L, int32_t* draft_tokens_dev, int32_t* draft_len_dev,
                          int32_t* source_dev, const int32_t* aux_tokens_dev, const int32_t* aux_len_dev,
                          void* stream);
+
+/* ---- tree drafts from the static automaton --------------------------------------------------- */
+
+/* Best-first tree draft over the top-k successors (Algorithm 5, with freq and top-k successors as in
+ * Appendix A.1/A.2; the automaton must have been built with tree_topk >= k).  For slot i the queue
+ * starts with (probability 1, states_dev[i], start_tokens_dev[i]); the most probable entry is
+ * popped and appended until max_size nodes are out or the queue is empty; a popped node pushes its
+ * k most frequent successors (freq descending, token ascending) with probability
+ * p * (freq(successor) / freq(state)) in IEEE float32 (quotient rounded first).  Among equal
+ * probabilities the entry pushed earlier is popped first.
+ *   states_dev        device int32 [B]   static state ids (sam_step's state[:, 0]); <= 0 gives an empty tree
+ *   start_tokens_dev  device int32 [B]   the token of node 0 (the last accepted token)
+ *   max_size 1..128, k 1..tree_topk
+ *   tree_tokens_dev   device int32 [B, max_size]  tokens in pop order, -1 beyond tree_size
+ *   tree_parents_dev  device int32 [B, max_size]  index of each node's parent, -1 for node 0 and beyond
+ *   tree_probs_dev    device float [B, max_size]  path probabilities; may be NULL
+ *   tree_size_dev     device int32 [B]
+ * Asynchronous on `stream`.  Errors: ARG (no tree data, k too large, sizes), CUDA. */
+int sam_tree_draft(const sam_static_t* st, int32_t batch, const int32_t* states_dev,
+                   const int32_t* start_tokens_dev, int32_t max_size, int32_t k,
+                   int32_t* tree_tokens_dev, int32_t* tree_parents_dev, float* tree_probs_dev,
+                   int32_t* tree_size_dev, void* stream);
+
+/* Copy freq (occurrences of each state's substrings in the corpus) of the first max_states states to
+ * the host (synchronous; inspection and tests).  Errors: ARG (no tree data), CUDA. */
+int sam_static_freq(const sam_static_t* st, uint32_t* freq_host, int64_t max_states);
 
 /* ---- retrieval without any allocation ------------------------------------------------------ */
 

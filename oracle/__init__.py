@@ -59,6 +59,9 @@ def _load():
     lib.osam_edges.argtypes = [vp, i32, _i32p, _i32p]
     lib.osam_tables.argtypes = [vp, _i32p, _i32p, _i32p, _i32p]
     lib.osam_counters.argtypes = [vp, _i64p]
+    lib.osam_freq.argtypes = [vp, _i64p]
+    lib.osam_topk.restype = i32
+    lib.osam_topk.argtypes = [vp, _i64p, i32, i32, _i32p, _i32p]
     lib.obatch_new.restype = vp
     lib.obatch_new.argtypes = [vp, _i32p, i64, i32, i32, i32, i32, i32, i32]
     lib.obatch_free.argtypes = [vp]
@@ -165,6 +168,19 @@ class Sam:
         c = (ctypes.c_int64 * 4)()
         self._lib.osam_counters(self._h, c)
         return dict(walk_inserts=c[0], clones=c[1], copied_edges=c[2], redirects=c[3])
+
+    def freq(self) -> np.ndarray:
+        """freq of every state (Appendix A.1/A.2): occurrences of its substrings in the text."""
+        f = np.zeros(self.n_states, dtype=np.int64)
+        self._lib.osam_freq(self._h, f.ctypes.data_as(_i64p))
+        return f
+
+    def topk(self, freq: np.ndarray, s: int, k: int):
+        """Top-k successors of s by freq: list of (token, target)."""
+        toks = np.empty(max(k, 1), dtype=np.int32)
+        tgts = np.empty(max(k, 1), dtype=np.int32)
+        n = self._lib.osam_topk(self._h, freq.ctypes.data_as(_i64p), int(s), int(k), _p32(toks), _p32(tgts))
+        return [(int(toks[i]), int(tgts[i])) for i in range(n)]
 
 
 class StepOut:

@@ -42,6 +42,7 @@ typedef struct {
     oedge_t** next;          /* next[s]: sorted array of deg[s] pairs */
     int32_t* deg;
     int32_t* cap;
+    uint8_t* is_clone;       /* 1 for states made by cloning (freq starts at 0), Appendix A.1 */
     int64_t n_states, cap_states;
     int64_t n_transitions;
     int32_t last;
@@ -97,6 +98,7 @@ static int grow_states(osam_t* S, int64_t want) {
     oedge_t** d = (oedge_t**)realloc(S->next, sizeof(oedge_t*) * (size_t)nc);     if (!d) return -1; S->next = d;
     int32_t* e = (int32_t*)realloc(S->deg, sizeof(int32_t) * (size_t)nc);         if (!e) return -1; S->deg = e;
     int32_t* f = (int32_t*)realloc(S->cap, sizeof(int32_t) * (size_t)nc);         if (!f) return -1; S->cap = f;
+    uint8_t* g = (uint8_t*)realloc(S->is_clone, (size_t)nc);                      if (!g) return -1; S->is_clone = g;
     S->cap_states = nc;
     return 0;
 }
@@ -106,7 +108,7 @@ static int32_t expand_state(osam_t* S, int32_t link, int32_t length, int32_t pos
     if (grow_states(S, S->n_states + 1)) { S->err = 1; return -1; }
     int32_t s = (int32_t)S->n_states++;
     S->link[s] = link; S->length[s] = length; S->min_endpos[s] = pos;
-    S->next[s] = NULL; S->deg[s] = 0; S->cap[s] = 0;
+    S->next[s] = NULL; S->deg[s] = 0; S->cap[s] = 0; S->is_clone[s] = 0;
     return s;
 }
 
@@ -123,7 +125,7 @@ osam_t* osam_new(int64_t states_hint) {
 void osam_free(osam_t* S) {
     if (!S) return;
     for (int64_t s = 0; s < S->n_states; s++) free(S->next[s]);
-    free(S->link); free(S->length); free(S->min_endpos); free(S->next); free(S->deg); free(S->cap);
+    free(S->link); free(S->length); free(S->min_endpos); free(S->next); free(S->deg); free(S->cap); free(S->is_clone);
     free(S);
 }
 
@@ -148,6 +150,7 @@ void osam_expand(osam_t* S, int32_t t) {
         } else {
             int32_t cl = expand_state(S, -1, -1, -1);
             if (cl < 0) return;
+            S->is_clone[cl] = 1;
             S->link[cl] = S->link[q];
             for (int i = 0; i < S->deg[q]; i++) {               /* cl.next = copy of q.next */
                 next_set(S, cl, S->next[q][i].tok, S->next[q][i].tgt);
@@ -217,6 +220,50 @@ void osam_tables(const osam_t* S, int32_t* link, int32_t* length, int32_t* min_e
 /* counters: walk_inserts, clones, copied_edges, redirects */
 void osam_counters(const osam_t* S, int64_t* out) {
     out[0] = S->c_walk_inserts; out[1] = S->c_clones; out[2] = S->c_copied_edges; out[3] = S->c_redirects;
+}
+
+/* ------------------------------------------------------------------ frequencies and top-k successors
+ *
+ * Appendix A.1 / A.2: every state carries `freq`, the frequency of occurrence of its substrings in
+ * the reference text, initialised to 1 for states made by expansion and 0 for clones; the top-k
+ * successors of a state are its transitions with the largest freq, and the transition probability
+ * is freq(target) / freq(state).
+ * Reading taken for the accumulation: freq(s) = init(s) + sum of freq(u) over the states u whose
+ * suffix link is s, i.e. the number of end positions of s's substrings.  (The printed recursion
+ * over `next` visits a state once per path that reaches it; the prose fixes the meaning.)
+ * Which states are clones is recorded when Expand makes them.
+ */
+void osam_freq(const osam_t* S, int64_t* freq) {
+    int64_t n = S->n_states;
+    /* order states by decreasing length with a counting sort */
+    int32_t maxlen = S->max_length;
+    int64_t* bucket = (int64_t*)calloc((size_t)maxlen + 2, sizeof(int64_t));
+    int32_t* order = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+    for (int64_t s = 0; s < n; s++) bucket[S->length[s] + 1]++;
+    for (int32_t l = 0; l <= maxlen; l++) bucket[l + 1] += bucket[l];
+    for (int64_t s = 0; s < n; s++) order[bucket[S->length[s]]++] = (int32_t)s;
+    for (int64_t s = 0; s < n; s++) freq[s] = (s != 0 && S->is_clone[s] == 0) ? 1 : 0;
+    for (int64_t i = n - 1; i > 0; i--) {
+        int32_t s = order[i];
+        if (S->link[s] >= 0) freq[S->link[s]] += freq[s];
+    }
+    free(bucket); free(order);
+}
+
+/* top-k successors of state s by (freq descending, token ascending); returns how many */
+int32_t osam_topk(const osam_t* S, const int64_t* freq, int32_t s, int32_t k, int32_t* toks, int32_t* tgts) {
+    int32_t n = 0;
+    for (int i = 0; i < S->deg[s]; i++) {
+        int32_t t = S->next[s][i].tok, u = S->next[s][i].tgt;      /* tokens come in ascending order */
+        int32_t pos = n;
+        while (pos > 0 && freq[tgts[pos - 1]] < freq[u]) pos--;     /* strictly larger moves ahead: ties keep token order */
+        if (pos >= k) continue;
+        int32_t last = n < k ? n : k - 1;
+        for (int32_t j = last; j > pos; j--) { toks[j] = toks[j - 1]; tgts[j] = tgts[j - 1]; }
+        toks[pos] = t; tgts[pos] = u;
+        if (n < k) n++;
+    }
+    return n;
 }
 
 /* ------------------------------------------------------------------ batched step

@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsamdraft.so")
-SOURCES = ["static_builder.cpp", "static_store.cu", "batch.cu", "step.cu", "probes.cu", "noalloc.cu", "accept.cu"]
+SOURCES = ["static_builder.cpp", "static_store.cu", "batch.cu", "step.cu", "probes.cu", "noalloc.cu", "accept.cu", "tree.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "--cudart", "shared"]
 

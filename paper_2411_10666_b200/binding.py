@@ -32,13 +32,14 @@ class SamError(RuntimeError):
 
 
 class BuildOpts(Structure):
-    _fields_ = [("hash_load", c_double), ("keep_host_copy", c_int32)]
+    _fields_ = [("hash_load", c_double), ("keep_host_copy", c_int32), ("tree_topk", c_int32)]
 
 
 class StaticInfo(Structure):
     _fields_ = [("n_tokens", c_int64), ("n_states", c_int64), ("n_transitions", c_int64),
                 ("n_hash_edges", c_int64), ("hash_buckets", c_int64), ("hash_max_probe", c_int32),
-                ("vocab", c_int32), ("device_bytes", c_size_t), ("build_seconds", c_double)]
+                ("vocab", c_int32), ("device_bytes", c_size_t), ("build_seconds", c_double),
+                ("tree_topk", c_int32), ("reserved", c_int32)]
 
 
 class BatchOpts(Structure):
@@ -78,6 +79,9 @@ SIGNATURES = {
     "sam_accept_greedy": (c_int, [c_int32, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32,
                                   c_void_p, c_void_p, c_void_p]),
     "sam_select_auxiliary": (c_int, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "sam_tree_draft": (c_int, [c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                               c_void_p, c_void_p]),
+    "sam_static_freq": (c_int, [c_void_p, c_void_p, c_int64]),
     "sam_retrieve_noalloc": (c_int, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32,
                                      c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "sam_noalloc_capacity_bytes": (c_size_t, []),
@@ -131,9 +135,9 @@ def _stream_ptr(stream=None):
 # thin wrappers, one per C call
 # ---------------------------------------------------------------------------------------------
 
-def sam_build_static(corpus_host, vocab: int, device: int = 0, hash_load: float = 0.0):
+def sam_build_static(corpus_host, vocab: int, device: int = 0, hash_load: float = 0.0, tree_topk: int = 0):
     corpus = _np32(corpus_host)
-    opts = BuildOpts(hash_load, 0)
+    opts = BuildOpts(hash_load, 0, tree_topk)
     h = c_void_p()
     _check(lib().sam_build_static(corpus.ctypes.data, corpus.shape[0], vocab, device, byref(opts), byref(h)),
            "sam_build_static")
@@ -291,6 +295,26 @@ def sam_select_auxiliary(draft_tokens, draft_len, source, aux_tokens, aux_len, s
                                       _dev_ptr(aux_len, "aux_len"), _stream_ptr(stream)), "sam_select_auxiliary")
 
 
+def sam_tree_draft(static_h, states, start_tokens, max_size: int, k: int, tree_tokens, tree_parents, tree_probs,
+                   tree_size, stream=None):
+    import torch
+    pp = None
+    if tree_probs is not None:
+        assert tree_probs.is_cuda and tree_probs.dtype == torch.float32 and tree_probs.is_contiguous()
+        pp = tree_probs.data_ptr()
+    _check(lib().sam_tree_draft(static_h, states.shape[0], _dev_ptr(states, "states"),
+                                _dev_ptr(start_tokens, "start_tokens"), max_size, k,
+                                _dev_ptr(tree_tokens, "tree_tokens"), _dev_ptr(tree_parents, "tree_parents"), pp,
+                                _dev_ptr(tree_size, "tree_size"), _stream_ptr(stream)), "sam_tree_draft")
+
+
+def sam_static_freq(h):
+    n = sam_static_info(h).n_states
+    out = np.empty(n, dtype=np.uint32)
+    _check(lib().sam_static_freq(h, out.ctypes.data, n), "sam_static_freq")
+    return out
+
+
 def sam_retrieve_noalloc(static_h, vocab, tokens, counts, L, l_bias, min_match,
                          draft_tokens, draft_len, match_len, source, state, status, stream=None):
     """One-shot retrieval over the library's built-in scratch array; allocates nothing."""
@@ -327,8 +351,8 @@ class StaticSam:
         self.handle, self.device = handle, device
 
     @classmethod
-    def build(cls, corpus, vocab: int, device: int = 0, hash_load: float = 0.0):
-        return cls(sam_build_static(corpus, vocab, device, hash_load), device)
+    def build(cls, corpus, vocab: int, device: int = 0, hash_load: float = 0.0, tree_topk: int = 0):
+        return cls(sam_build_static(corpus, vocab, device, hash_load, tree_topk), device)
 
     @classmethod
     def load(cls, path: str, device: int = 0):

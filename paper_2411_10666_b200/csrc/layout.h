@@ -13,6 +13,9 @@
 //               hash(state, tok) & mask, overflow goes to the following buckets.  An empty entry
 //               has state == SAM_NONE; a bucket with an empty entry ends a probe sequence.
 //   corpus    : the int32 token text, padded so vector reads past the end stay in bounds.
+//   freq, topk: optional, for tree drafts — the occurrence count of every state, and for states
+//               with hashed transitions their k most frequent successors (a state with at most two
+//               transitions has them all in its record).
 //
 // DYNAMIC automata (one per sequence slot, written by the slot's own warp only)
 //   rec       : 32 bytes per state, in slabs from the shared pool, addressed through the slot's
@@ -64,6 +67,11 @@ struct SamStaticRec {   // 32 bytes
 
 struct SamHashEnt { uint32_t state, tok, tgt, pad; };   // 16 bytes
 
+#define SAM_TOPK_MAX 6
+// Top-k successors of a state with hashed transitions (freq descending, token ascending): 64 bytes.
+// Kept in an open-addressing table keyed by state (linear probing, state == SAM_NONE is empty).
+struct SamTopkEnt { uint32_t state, n, pad0, pad1; uint32_t tok[SAM_TOPK_MAX]; uint32_t tgt[SAM_TOPK_MAX]; };
+
 // 64-bit multiplicative mix of (state, token); upper half is the hash.
 SAM_HD uint32_t sam_hash2(uint32_t state, uint32_t tok) {
     uint64_t k = ((uint64_t)state << 32) | tok;
@@ -91,6 +99,11 @@ struct SamStaticView {
     int32_t vocab;
     int64_t n_tokens;
     int64_t n_states;
+    // tree drafts (present when the automaton was built with tree_topk > 0)
+    const uint32_t* freq;     // occurrences of each state's substrings in the corpus
+    const uint4* topk;        // SamTopkEnt table, four 16-byte words per entry
+    uint32_t topk_mask;       // entries - 1
+    int32_t tree_k;           // successors kept per hashed state (0: no tree data)
 };
 
 // Device-side view of a batch workspace.

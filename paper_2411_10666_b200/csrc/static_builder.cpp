@@ -14,8 +14,10 @@
 
 #include <sys/mman.h>
 #include <chrono>
+#include <algorithm>
 #include <cstring>
 #include <new>
+#include <utility>
 
 namespace {
 
@@ -71,7 +73,7 @@ private:
 class Builder {
 public:
     Builder(SamStaticRec* rec, int64_t cap, int32_t vocab)
-        : rec_(rec), cap_(cap), root_(vocab, SAM_NONE) {
+        : rec_(rec), cap_(cap), root_(vocab, SAM_NONE), clone_((size_t)(cap / 64 + 1), 0) {
         new_state(0, 0);
         rec_[0].link = SAM_NONE;
     }
@@ -94,6 +96,7 @@ public:
             rec_[c].link = q;
         } else {
             uint32_t cl = new_state(rec_[p].len + 1, rec_[q].min_endpos);
+            clone_[cl >> 6] |= 1ull << (cl & 63);
             copy_edges(q, cl);
             rec_[cl].link = rec_[q].link;
             while (p >= 0 && find((uint32_t)p, t) == q) {
@@ -112,6 +115,19 @@ public:
     int64_t n_ovf() const { return n_ovf_; }
     std::vector<uint32_t>& root() { return root_; }
     const OvfTable& ovf() const { return ovf_; }
+    bool is_clone(int64_t s) const { return (clone_[(size_t)(s >> 6)] >> (s & 63)) & 1; }
+    // every transition of a state with hashed transitions: the two inline ones and the threaded list
+    void edges_of(uint32_t s, std::vector<std::pair<uint32_t, uint32_t>>& out) {
+        out.clear();
+        const SamStaticRec& r = rec_[s];
+        if (r.deg >= 1) out.emplace_back(r.tok0, r.tgt0 & SAM_IDMASK);
+        if (r.deg >= 2) out.emplace_back(r.tok1, r.tgt1 & SAM_IDMASK);
+        if (r.deg > 2) {
+            OvfEnt* h = ovf_.find(s, HEAD_TOK);
+            uint32_t t = h ? h->tgt : SAM_NONE;
+            while (t != SAM_NONE) { OvfEnt* e = ovf_.find(s, t); out.emplace_back(t, e->tgt & SAM_IDMASK); t = e->next_tok; }
+        }
+    }
 
 private:
     SamStaticRec* rec_;
@@ -120,6 +136,7 @@ private:
     int32_t n_text_ = 0;
     int64_t last_ = 0;
     std::vector<uint32_t> root_;
+    std::vector<uint64_t> clone_;     // bit s: state s was made by cloning
     OvfTable ovf_;
 
     uint32_t new_state(int32_t len, int32_t endpos) {
@@ -187,9 +204,11 @@ SamHostImage::~SamHostImage() {
     if (rec) munmap(rec, rec_map_bytes);
 }
 
-int sam_host_build(const int32_t* corpus, int64_t n, int32_t vocab, double hash_load, SamHostImage* out) {
+int sam_host_build(const int32_t* corpus, int64_t n, int32_t vocab, double hash_load, int32_t tree_k,
+                   SamHostImage* out) {
     if (!corpus || n < 1 || vocab < 1 || !out) return SAM_ERR_ARG;
     if (n > (1ll << 30)) return SAM_ERR_LIMIT;          // state ids must fit 31 bits
+    if (tree_k < 0 || tree_k > SAM_TOPK_MAX) return SAM_ERR_ARG;
     if (!(hash_load > 0.0) || hash_load > 0.9) hash_load = 0.5;
     auto t0 = std::chrono::steady_clock::now();
 
@@ -259,6 +278,51 @@ int sam_host_build(const int32_t* corpus, int64_t n, int32_t vocab, double hash_
             }
             if (ok) { out->hash_mask = mask; out->hash_max_probe = max_probe; break; }
             buckets <<= 1;                                 // pathological clustering: halve the load
+        }
+
+        // Tree-draft data (Appendix A.1/A.2): freq = occurrences of a state's substrings, 1 for a
+        // state made by expansion and 0 for a clone, summed over the suffix-link tree from the
+        // longest states down; then the k most frequent successors of every state whose
+        // transitions are hashed (freq descending, token ascending).
+        out->tree_k = tree_k;
+        if (tree_k > 0) {
+            std::vector<uint32_t>& freq = out->freq;
+            freq.assign((size_t)ns, 0);
+            std::vector<uint32_t> start((size_t)n + 2, 0), order((size_t)ns);
+            for (int64_t s = 0; s < ns; s++) start[(size_t)rec[s].len + 1]++;
+            for (int64_t l = 0; l <= n; l++) start[(size_t)l + 1] += start[(size_t)l];
+            for (int64_t s = 0; s < ns; s++) order[start[(size_t)rec[s].len]++] = (uint32_t)s;
+            for (int64_t s = 1; s < ns; s++) freq[(size_t)s] = b.is_clone(s) ? 0u : 1u;
+            for (int64_t i = ns - 1; i > 0; i--) {
+                uint32_t s = order[(size_t)i];
+                freq[rec[s].link & SAM_IDMASK] += freq[s];
+            }
+            int64_t hashed = 0;
+            for (int64_t s = 1; s < ns; s++) hashed += rec[s].deg > 2;
+            uint64_t cap_t = 16;
+            while (cap_t < (uint64_t)hashed * 2) cap_t <<= 1;
+            SamTopkEnt empty;
+            memset(&empty, 0, sizeof(empty));
+            empty.state = SAM_NONE;
+            out->topk.assign((size_t)cap_t, empty);
+            out->topk_mask = (uint32_t)(cap_t - 1);
+            std::vector<std::pair<uint32_t, uint32_t>> ed;
+            for (int64_t s = 1; s < ns; s++) {
+                if (rec[s].deg <= 2) continue;
+                b.edges_of((uint32_t)s, ed);
+                size_t keep = std::min<size_t>((size_t)tree_k, ed.size());
+                std::partial_sort(ed.begin(), ed.begin() + keep, ed.end(),
+                                  [&](const std::pair<uint32_t, uint32_t>& x, const std::pair<uint32_t, uint32_t>& y) {
+                                      if (freq[x.second] != freq[y.second]) return freq[x.second] > freq[y.second];
+                                      return x.first < y.first;
+                                  });
+                SamTopkEnt e = empty;
+                e.state = (uint32_t)s; e.n = (uint32_t)keep;
+                for (size_t j = 0; j < keep; j++) { e.tok[j] = ed[j].first; e.tgt[j] = flagged(ed[j].second); }
+                uint32_t at = sam_hash1((uint32_t)s) & out->topk_mask;
+                while (out->topk[at].state != SAM_NONE) at = (at + 1) & out->topk_mask;
+                out->topk[at] = e;
+            }
         }
     } catch (const std::bad_alloc&) {
         return SAM_ERR_NOMEM;

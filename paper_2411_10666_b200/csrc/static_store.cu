@@ -12,7 +12,7 @@ namespace {
 thread_local int g_last_cuda = 0;
 
 constexpr uint64_t FILE_MAGIC = 0x314D41534D415353ull;   // "SSAMSAM1"
-constexpr uint32_t FILE_VERSION = 1;
+constexpr uint32_t FILE_VERSION = 2;
 constexpr size_t CORPUS_PAD_TOKENS = 64;                  // vector reads past the end stay in bounds
 
 struct FileHeader {
@@ -20,7 +20,8 @@ struct FileHeader {
     uint32_t version, vocab;
     int64_t n_tokens, n_states, n_transitions, n_hash_edges, hash_buckets;
     int32_t hash_max_probe, pad;
-    uint64_t len_rec, len_root, len_hash, len_corpus;
+    uint64_t len_rec, len_root, len_hash, len_corpus, len_freq, len_topk;
+    int32_t tree_k, pad2;
     uint64_t checksum;
 };
 
@@ -37,6 +38,8 @@ void layout_sections(sam_static* st) {
     st->off_root = off;   off = sam_align_up(off + st->len_root, 256);
     st->off_hash = off;   off = sam_align_up(off + st->len_hash, 256);
     st->off_corpus = off; off = sam_align_up(off + st->len_corpus, 256);
+    st->off_freq = off;   off = sam_align_up(off + st->len_freq, 256);
+    st->off_topk = off;   off = sam_align_up(off + st->len_topk, 256);
     st->dev_bytes = off;
 }
 
@@ -51,6 +54,10 @@ void make_view(sam_static* st) {
     st->view.vocab = st->info.vocab;
     st->view.n_tokens = st->info.n_tokens;
     st->view.n_states = st->info.n_states;
+    st->view.freq = (const uint32_t*)(base + st->off_freq);
+    st->view.topk = (const uint4*)(base + st->off_topk);
+    st->view.topk_mask = st->len_topk ? (uint32_t)(st->len_topk / sizeof(SamTopkEnt) - 1) : 0;
+    st->view.tree_k = st->info.tree_topk;
 }
 
 // collect the transitions of one state: inline ones, hashed ones, or the root row
@@ -113,13 +120,13 @@ extern "C" int sam_build_static(const int32_t* corpus_host, int64_t n_tokens, in
     if (!out) return SAM_ERR_ARG;
     *out = nullptr;
     if (!corpus_host || n_tokens < 1 || vocab < 1) return SAM_ERR_ARG;
-    if (opts && opts->keep_host_copy != 0) return SAM_ERR_ARG;
+    if (opts && (opts->keep_host_copy != 0 || opts->tree_topk < 0 || opts->tree_topk > SAM_TOPK_MAX)) return SAM_ERR_ARG;
     if (n_tokens > (1ll << 30)) return SAM_ERR_LIMIT;
     int rc = check_device(device);
     if (rc) return rc;
 
     SamHostImage img;
-    rc = sam_host_build(corpus_host, n_tokens, vocab, opts ? opts->hash_load : 0.0, &img);
+    rc = sam_host_build(corpus_host, n_tokens, vocab, opts ? opts->hash_load : 0.0, opts ? opts->tree_topk : 0, &img);
     if (rc) return rc;
 
     sam_static* st = new (std::nothrow) sam_static();
@@ -138,6 +145,9 @@ extern "C" int sam_build_static(const int32_t* corpus_host, int64_t n_tokens, in
     st->len_root = sam_align_up((size_t)vocab * 4, 8);
     st->len_hash = img.hash.size() * sizeof(SamHashEnt);
     st->len_corpus = sam_align_up(((size_t)n_tokens + CORPUS_PAD_TOKENS) * 4, 8);
+    st->info.tree_topk = img.tree_k;
+    st->len_freq = sam_align_up(img.freq.size() * 4, 8);
+    st->len_topk = img.topk.size() * sizeof(SamTopkEnt);
     layout_sections(st);
     st->info.device_bytes = st->dev_bytes;
 
@@ -151,6 +161,8 @@ extern "C" int sam_build_static(const int32_t* corpus_host, int64_t n_tokens, in
     if (e == cudaSuccess) e = cudaMemcpy(base + st->off_root, img.root_row.data(), (size_t)vocab * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(base + st->off_hash, img.hash.data(), st->len_hash, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(base + st->off_corpus, corpus_host, (size_t)n_tokens * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !img.freq.empty()) e = cudaMemcpy(base + st->off_freq, img.freq.data(), img.freq.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !img.topk.empty()) e = cudaMemcpy(base + st->off_topk, img.topk.data(), st->len_topk, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { sam_set_cuda_error(e); cudaFree(st->dev_base); delete st; return SAM_ERR_CUDA; }
     make_view(st);
     *out = st;
@@ -183,15 +195,16 @@ extern "C" int sam_static_save(const sam_static_t* st, const char* path) {
     h.n_transitions = st->info.n_transitions; h.n_hash_edges = st->info.n_hash_edges;
     h.hash_buckets = st->info.hash_buckets; h.hash_max_probe = st->info.hash_max_probe;
     h.len_rec = st->len_rec; h.len_root = st->len_root; h.len_hash = st->len_hash; h.len_corpus = st->len_corpus;
+    h.len_freq = st->len_freq; h.len_topk = st->len_topk; h.tree_k = st->info.tree_topk;
     int rc = SAM_OK;
     if (fwrite(&h, sizeof(h), 1, f) != 1) rc = SAM_ERR_IO;
     const size_t CHUNK = 64u << 20;
     std::vector<char> buf;
     try { buf.resize(CHUNK); } catch (const std::bad_alloc&) { fclose(f); return SAM_ERR_NOMEM; }
     uint64_t sum = 0xCBF29CE484222325ull;
-    const size_t offs[4] = {st->off_rec, st->off_root, st->off_hash, st->off_corpus};
-    const size_t lens[4] = {st->len_rec, st->len_root, st->len_hash, st->len_corpus};
-    for (int s = 0; s < 4 && rc == SAM_OK; s++) {
+    const size_t offs[6] = {st->off_rec, st->off_root, st->off_hash, st->off_corpus, st->off_freq, st->off_topk};
+    const size_t lens[6] = {st->len_rec, st->len_root, st->len_hash, st->len_corpus, st->len_freq, st->len_topk};
+    for (int s = 0; s < 6 && rc == SAM_OK; s++) {
         for (size_t done = 0; done < lens[s] && rc == SAM_OK; done += CHUNK) {
             size_t n = lens[s] - done < CHUNK ? lens[s] - done : CHUNK;
             cudaError_t e = cudaMemcpy(buf.data(), (char*)st->dev_base + offs[s] + done, n, cudaMemcpyDeviceToHost);
@@ -223,7 +236,12 @@ extern "C" int sam_static_load(const char* path, int device, sam_static_t** out)
                 h.len_rec == (uint64_t)h.n_states * sizeof(SamStaticRec) &&
                 h.len_root == sam_align_up((size_t)h.vocab * 4, 8) &&
                 h.len_hash == (uint64_t)h.hash_buckets * SAM_HASH_BUCKET * sizeof(SamHashEnt) &&
-                h.len_corpus == sam_align_up(((size_t)h.n_tokens + CORPUS_PAD_TOKENS) * 4, 8);
+                h.len_corpus == sam_align_up(((size_t)h.n_tokens + CORPUS_PAD_TOKENS) * 4, 8) &&
+                h.tree_k >= 0 && h.tree_k <= SAM_TOPK_MAX &&
+                (h.tree_k == 0 ? (h.len_freq == 0 && h.len_topk == 0)
+                               : (h.len_freq == sam_align_up((size_t)h.n_states * 4, 8) && h.len_topk >= sizeof(SamTopkEnt) &&
+                                  h.len_topk % sizeof(SamTopkEnt) == 0 &&
+                                  ((h.len_topk / sizeof(SamTopkEnt)) & (h.len_topk / sizeof(SamTopkEnt) - 1)) == 0));
     if (!sane) { fclose(f); return SAM_ERR_FORMAT; }
 
     sam_static* st = new (std::nothrow) sam_static();
@@ -234,6 +252,7 @@ extern "C" int sam_static_load(const char* path, int device, sam_static_t** out)
     st->info.n_hash_edges = h.n_hash_edges; st->info.hash_buckets = h.hash_buckets;
     st->info.hash_max_probe = h.hash_max_probe; st->info.vocab = (int32_t)h.vocab;
     st->len_rec = h.len_rec; st->len_root = h.len_root; st->len_hash = h.len_hash; st->len_corpus = h.len_corpus;
+    st->len_freq = h.len_freq; st->len_topk = h.len_topk; st->info.tree_topk = h.tree_k;
     layout_sections(st);
     st->info.device_bytes = st->dev_bytes;
 
@@ -246,10 +265,10 @@ extern "C" int sam_static_load(const char* path, int device, sam_static_t** out)
     std::vector<char> buf;
     try { buf.resize(CHUNK); } catch (const std::bad_alloc&) { cudaFree(st->dev_base); delete st; fclose(f); return SAM_ERR_NOMEM; }
     uint64_t sum = 0xCBF29CE484222325ull;
-    const size_t offs[4] = {st->off_rec, st->off_root, st->off_hash, st->off_corpus};
-    const size_t lens[4] = {st->len_rec, st->len_root, st->len_hash, st->len_corpus};
+    const size_t offs[6] = {st->off_rec, st->off_root, st->off_hash, st->off_corpus, st->off_freq, st->off_topk};
+    const size_t lens[6] = {st->len_rec, st->len_root, st->len_hash, st->len_corpus, st->len_freq, st->len_topk};
     rc = SAM_OK;
-    for (int s = 0; s < 4 && rc == SAM_OK; s++) {
+    for (int s = 0; s < 6 && rc == SAM_OK; s++) {
         for (size_t done = 0; done < lens[s] && rc == SAM_OK; done += CHUNK) {
             size_t n = lens[s] - done < CHUNK ? lens[s] - done : CHUNK;
             if (fread(buf.data(), 1, n, f) != n) { rc = SAM_ERR_FORMAT; break; }
@@ -338,7 +357,7 @@ extern "C" int sam_build_static_tables(const int32_t* corpus_host, int64_t n_tok
                                        int32_t* edge_src, int32_t* edge_tok, int32_t* edge_tgt, int64_t max_edges) {
     if (!n_states || !n_transitions) return SAM_ERR_ARG;
     SamHostImage img;
-    int rc = sam_host_build(corpus_host, n_tokens, vocab, 0.0, &img);
+    int rc = sam_host_build(corpus_host, n_tokens, vocab, 0.0, 0, &img);
     if (rc) return rc;
     *n_states = img.n_states;
     *n_transitions = img.n_transitions;
@@ -384,4 +403,14 @@ extern "C" int sam_build_static_tables(const int32_t* corpus_host, int64_t n_tok
     }
     if (k != img.n_transitions) rc = SAM_ERR_FORMAT;
     return rc;
+}
+
+extern "C" int sam_static_freq(const sam_static_t* st, uint32_t* freq_host, int64_t max_states) {
+    if (!st || !freq_host || max_states < 0) return SAM_ERR_ARG;
+    if (st->info.tree_topk <= 0) return SAM_ERR_ARG;
+    SamDeviceGuard guard(st->device);
+    if (!guard.ok) return SAM_ERR_CUDA;
+    int64_t n = st->info.n_states < max_states ? st->info.n_states : max_states;
+    SAM_CUDA(cudaMemcpy(freq_host, st->view.freq, (size_t)n * 4, cudaMemcpyDeviceToHost));
+    return SAM_OK;
 }
