@@ -269,6 +269,9 @@ def main_ours(args):
     ct_pin = torch.from_numpy(counts).pin_memory()
     mk = lambda *s: torch.empty(s, dtype=torch.int32).pin_memory()
     ho = [mk(B, L), mk(B), mk(B, 2), mk(B), mk(B, 2), mk(B)]
+    ho_ptr = [t.data_ptr() for t in ho]                     # addresses are passed as plain ints
+    nt_base, nt_step = nt_pin.data_ptr(), B * spec.accept_max * 4
+    ct_base, ct_step = ct_pin.data_ptr(), B * 4
     e2e_times = []
     for _ in range(3):
         prepare()
@@ -276,8 +279,8 @@ def main_ours(args):
         if world > 1:
             torch.distributed.barrier()
         t1 = time.perf_counter()
-        for s in range(Wm, Wm + K):
-            sd.sam_step_host(batch.handle, nt_pin[s], spec.accept_max, ct_pin[s], L, *ho)
+        for s in range(Wm, Wm + K):                     # step s reads its own rows of the pinned arrays
+            sd.sam_step_host(batch.handle, nt_base + s * nt_step, spec.accept_max, ct_base + s * ct_step, L, *ho_ptr)
         torch.cuda.synchronize()
         e2e_times.append((time.perf_counter() - t1) * 1e3)
     clocks = sampler.stop() if sampler else None

@@ -242,10 +242,11 @@ def sam_run_steps(h, new_tokens, stride, counts, n_steps, L, out_per_step,
 
 
 def _host_ptr(t, name):
-    """Host buffer: a numpy int32 array or a CPU (ideally pinned) int32 torch tensor."""
+    """Host buffer: a numpy int32 array, a CPU (ideally pinned) int32 torch tensor, or a plain int
+    that is taken as the buffer's address (for loops that precompute their pointers)."""
+    if t is None or isinstance(t, int):
+        return t
     import torch
-    if t is None:
-        return None
     if isinstance(t, np.ndarray):
         assert t.dtype == np.int32 and t.flags["C_CONTIGUOUS"], name
         return t.ctypes.data

@@ -2,6 +2,7 @@
 // the host-array step, the step replay loop and the inspection calls.
 #include "common.h"
 
+#include <chrono>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -9,6 +10,7 @@
 namespace {
 
 constexpr size_t SAM_ZERO_COPY_MAX_BYTES = 256u << 10;   // larger host steps go through two DMA copies
+constexpr int SAM_POLL_LIMIT_US = 2000;                  // how long a host step polls its completion flag
 
 struct WsLayout {
     size_t off_hdr, off_ctrl, off_free, off_owner, off_reset, off_text, off_root, off_stage, off_pool, total;
@@ -68,7 +70,7 @@ __global__ void init_pool_kernel(SamBatchView W) {
         W.slab_owner[s] = -1;
     }
     for (size_t b = i; b < (size_t)W.batch; b += stride) W.reset_flag[b] = 0;
-    if (i == 0) { W.pool_hdr[0] = W.pool_slabs; W.pool_hdr[1] = W.pool_slabs; }
+    if (i == 0) { W.pool_hdr[0] = W.pool_slabs; W.pool_hdr[1] = W.pool_slabs; W.pool_hdr[4] = 0; }
 }
 
 // slots == nullptr: every slot.  Clears control blocks and root tables and raises reset flags.
@@ -249,7 +251,7 @@ extern "C" int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* 
 
     SamDeviceGuard guard(b->device);
     if (!guard.ok) { delete b; return SAM_ERR_CUDA; }
-    e = cudaHostAlloc((void**)&b->host_stage, w.stage_words * 4, cudaHostAllocMapped);
+    e = cudaHostAlloc((void**)&b->host_stage, (w.stage_words + 16) * 4, cudaHostAllocMapped);   // + the completion flag
     if (e == cudaSuccess) e = cudaHostGetDevicePointer((void**)&b->host_stage_dev, b->host_stage, 0);
     if (e != cudaSuccess) {
         sam_set_cuda_error(e); cudaGetLastError();
@@ -257,6 +259,7 @@ extern "C" int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* 
         delete b;
         return SAM_ERR_NOMEM;
     }
+    b->host_stage[w.stage_words] = 0;
     cudaStream_t s = (cudaStream_t)stream;
     init_pool_kernel<<<296, 256, 0, s>>>(V);
     reset_slots_kernel<<<V.batch, 128, 0, s>>>(V, nullptr, V.batch);
@@ -362,10 +365,22 @@ extern "C" int sam_step_host(sam_batch_t* b, const int32_t* new_tokens_host, int
         // staging area directly; the bytes cross the bus inside the kernel instead of in two copies
         int32_t* zd = b->host_stage_dev;
         int32_t* zo = zd + in_words;
-        rc = sam_launch_step(b, zd, stride, zd + B * stride, L, zo, zo + B * L, zo + B * L + B, zo + B * L + 3 * B,
-                             zo + B * L + 4 * B, zo + B * L + 6 * B, s);
+        // completion: the last block writes this step's sequence number into the flag word behind the
+        // staging area; polling it costs less than a stream synchronisation.  The poll is bounded;
+        // past the bound (other work queued ahead on the stream, or a failed launch) it falls back.
+        volatile int32_t* flag = b->host_stage + b->stage_words;
+        const int32_t seq = ++b->host_seq == 0 ? ++b->host_seq : b->host_seq;
+        rc = sam_launch_step_signal(b, zd, stride, zd + B * stride, L, zo, zo + B * L, zo + B * L + B, zo + B * L + 3 * B,
+                                    zo + B * L + 4 * B, zo + B * L + 6 * B, s, b->host_stage_dev + b->stage_words, seq);
         if (rc) return rc;
-        SAM_CUDA(cudaStreamSynchronize(s));
+        const auto t0 = std::chrono::steady_clock::now();
+        bool seen = false;
+        for (uint32_t spin = 0;; spin++) {
+            if (*flag == seq) { seen = true; break; }
+            if ((spin & 1023u) == 1023u &&
+                std::chrono::steady_clock::now() - t0 > std::chrono::microseconds(SAM_POLL_LIMIT_US)) break;
+        }
+        if (!seen) SAM_CUDA(cudaStreamSynchronize(s));
     } else {
         SAM_CUDA(cudaMemcpyAsync(dev, hst, in_words * 4, cudaMemcpyHostToDevice, s));
         int32_t* o = dev + in_words;

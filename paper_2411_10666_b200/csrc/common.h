@@ -26,6 +26,7 @@ struct sam_batch {
     size_t stage_words;           // int32 words of device staging
     int32_t* host_stage;          // pinned, device-mapped host staging area
     int32_t* host_stage_dev;      // the same memory as the device addresses it
+    int32_t host_seq;             // sequence number of the last host-array step (completion flag value)
 };
 
 void sam_set_cuda_error(cudaError_t e);
@@ -53,6 +54,11 @@ static inline size_t sam_align_up(size_t x, size_t a) { return (x + a - 1) / a *
 int sam_launch_step(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
                     int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
                     int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream);
+
+int sam_launch_step_signal(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
+                           int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
+                           int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream,
+                           int32_t* done_flag_dev, int32_t done_seq);
 
 // helpers implemented in batch.cu
 int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBatchView* view,

@@ -27,6 +27,9 @@ struct StepArgs {
     const int32_t* new_tokens; int32_t stride; const int32_t* counts; int32_t L;
     int32_t* draft_tokens; int32_t* draft_len; int32_t* match_len; int32_t* source;
     int32_t* state; int32_t* status;
+    // optional completion signal for the host-array step: the last block to finish writes done_seq to
+    // *done_flag (host-mapped memory) so the host can poll instead of synchronising the stream
+    int32_t* done_count; int32_t* done_flag; int32_t done_seq;
 };
 
 // ------------------------------------------------------------------ draft read
@@ -479,6 +482,18 @@ __device__ __forceinline__ int dyn_fresh_run(Dyn& D, uint32_t tk, int j, int cnt
     return r;
 }
 
+// Called by one thread of a block after the block's outputs are written (and made known to that
+// thread by a block barrier where another warp wrote some of them).
+__device__ __forceinline__ void signal_done(const StepArgs& A) {
+    __threadfence_system();
+    const int prev = atomicAdd(A.done_count, 1);
+    if (prev == (int)gridDim.x - 1) {
+        *A.done_count = 0;
+        __threadfence_system();
+        *reinterpret_cast<volatile int32_t*>(A.done_flag) = A.done_seq;
+    }
+}
+
 // ------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ StepArgs A) {
     const int b = blockIdx.x;
@@ -525,6 +540,8 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                 if (A.state) { A.state[2 * b] = 0; A.state[2 * b + 1] = 0; }
                 A.status[b] = status;
             }
+            __syncwarp();
+            if (A.done_flag && lane == 0) signal_done(A);
         }
         return;
     }
@@ -673,6 +690,10 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         if (A.state) { A.state[2 * b] = any_err ? 0 : sh_s[0]; A.state[2 * b + 1] = any_err ? 0 : sh_s[1]; }
         A.status[b] = any_err;
     }
+    if (A.done_flag) {
+        __syncthreads();
+        if (threadIdx.x == 0) signal_done(A);
+    }
 }
 
 }  // namespace
@@ -680,7 +701,16 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
 int sam_launch_step(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
                     int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
                     int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream) {
+    return sam_launch_step_signal(b, new_tokens, stride, counts, L, draft_tokens, draft_len, match_len, source, state,
+                                  status, stream, nullptr, 0);
+}
+
+int sam_launch_step_signal(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
+                           int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
+                           int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream,
+                           int32_t* done_flag_dev, int32_t done_seq) {
     StepArgs A;
+    A.done_count = b->view.pool_hdr + 4; A.done_flag = done_flag_dev; A.done_seq = done_seq;
     A.has_static = b->st != nullptr;
     if (b->st) A.S = b->st->view;
     else { A.S = SamStaticView(); A.S.vocab = b->view.vocab; }
