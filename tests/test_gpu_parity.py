@@ -207,3 +207,62 @@ def test_full_size_configs(P, key):
     ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=os.cpu_count())
     assert_same(got, ref, key)
     assert st.info.n_states == S.n_states and st.info.n_transitions == S.n_transitions
+
+
+def test_runs_of_new_tokens_across_slabs_and_crowded_root_buckets(P):
+    """The parallel path for runs of new tokens: runs that straddle a slab boundary (4 KiB slabs hold
+    128 records), chunks with repeated tokens, and tiny root tables where many tokens share a bucket."""
+    rng = random.Random(77)
+    empty = lambda B: np.zeros((B, 0), np.int32)
+    # all-distinct text in steps of 24 (128 is not a multiple of 24) and of 100 (several chunks of 32)
+    for step in (24, 100):
+        n = 1000
+        x = list(range(n)); rng.shuffle(x)
+        rows = [x[i:i + step] + [-1] * (step - len(x[i:i + step])) for i in range(0, n, step)]
+        nt = np.array(rows, dtype=np.int32).reshape(len(rows), 1, step)
+        ct = np.array([min(step, n - i) for i in range(0, n, step)], dtype=np.int32).reshape(-1, 1)
+        ref, ob, _ = oracle_run(None, n, empty(1), nt, ct, 8, n)
+        got, batch = gpu_run(P, None, n, empty(1), nt, ct, 8, n, slab_bytes=4096)
+        assert_same(got, ref)
+        assert_dynamic_automata_equal(batch, ob, [0], n)
+    # short sequences (root table of 64 entries = 8 buckets): distinct tokens, then tokens with repeats
+    for case in range(120):
+        n = rng.randint(8, 32)
+        vocab = 100000
+        if case % 2 == 0:
+            x = rng.sample(range(vocab), n)
+        else:
+            pool = rng.sample(range(vocab), rng.randint(3, n))
+            x = [rng.choice(pool) for _ in range(n)]
+        B = 3
+        xs = [x, x[::-1], x[n // 2:] + x[:n // 2]]
+        k = rng.choice([n, 7, 32])
+        rows, cnts = [], []
+        for i in range(0, n, k):
+            rows.append([t[i:i + k] + [-1] * (k - len(t[i:i + k])) for t in xs]); cnts.append([min(k, n - i)] * B)
+        nt = np.array(rows, dtype=np.int32); ct = np.array(cnts, dtype=np.int32)
+        ref, ob, _ = oracle_run(None, vocab, empty(B), nt, ct, 4, n)
+        got, batch = gpu_run(P, None, vocab, empty(B), nt, ct, 4, n)
+        assert_same(got, ref, "case %d" % case)
+        assert_dynamic_automata_equal(batch, ob, range(B), n)
+
+
+def test_pool_exhaustion_leaves_other_slots_exact(P):
+    """When the shared pool runs dry some slots stop with status 1; the slots that did not stop still
+    agree with the oracle on everything."""
+    rng = random.Random(8)
+    vocab, n, L, B = 3000, 1200, 8, 6
+    nt = np.array([[rng.randrange(vocab) for _ in range(n)] for _ in range(B)], dtype=np.int32)
+    step = 60
+    rows = nt.reshape(B, n // step, step).transpose(1, 0, 2).copy()
+    ct = np.full((n // step, B), step, dtype=np.int32)
+    ref, _, _ = oracle_run(None, vocab, np.zeros((B, 0), np.int32), rows, ct, L, n)
+    got, _ = gpu_run(P, None, vocab, np.zeros((B, 0), np.int32), rows, ct, L, n, slab_bytes=4096, pool_slabs=40)
+    st = got["status"]
+    assert set(np.unique(st).tolist()) <= {0, 1} and (st[-1] == 1).any() and (st[0] == 0).all()
+    ok = st == 0
+    for k in ("draft_len", "match_len", "source", "state", "draft_tokens"):
+        assert np.array_equal(got[k][ok], ref[k][ok]), k
+    assert (got["draft_len"][~ok] == 0).all()
+    # once stopped, always stopped
+    assert (np.diff((st != 0).astype(int), axis=0) >= 0).all()
