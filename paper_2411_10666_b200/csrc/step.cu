@@ -8,11 +8,18 @@
 // the first end position of their state, fetch their candidate draft speculatively, and the
 // source rule l1 > l2 + l_bias (Section 3.2) picks which one is written out.
 //
-// Each warp runs one dependent chain of memory reads, so the work is latency-bound: every value
-// is warp-uniform (all lanes read the same 32-byte record, one request), and the lanes are used
-// side by side only where a structure is wide — a 128-byte hash bucket, a 256-byte root-table
-// bucket, an edge block, the draft read.  Independent reads are issued together (record + hash
-// bucket, root-row entries for all tokens of the step up front).
+// Each warp runs one dependent chain of memory reads, so the work is latency-bound, and the code
+// is organised around the number of read round trips per step:
+//   - everything a step needs to start (64 control words with copies of both match states'
+//     records, the count, the first 32 tokens) is read in one round trip;
+//   - values are warp-uniform (all lanes read the same 32-byte record: one request); lanes work
+//     side by side only where a structure is wide (a 128-byte hash bucket, a window of 32 root-table
+//     entries, an edge block, the draft read);
+//   - independent reads go out together: a static state's record with its hash bucket, the root-row
+//     entries of all tokens of the step, and the dynamic root-table lookups of all tokens of a chunk,
+//     one lane per token;
+//   - runs of tokens that are new to the sequence while nothing is matched are extended by the lanes
+//     in parallel (each such Expand is three independent writes).
 #include "common.h"
 
 namespace {
