@@ -60,6 +60,8 @@ def parse_args():
     ap.add_argument("--max-repeats", type=int, default=300)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probes", action="store_true")
+    ap.add_argument("--closed-loop", action="store_true",
+                    help="also run draft -> verify -> accept -> update on the device with the true continuation as target")
     return ap.parse_args()
 
 
@@ -157,6 +159,54 @@ def run_oracle_timed(spec, corpus, seqs, counts, new_tokens, steps_lo, steps_hi,
     c1 = ob.counters()
     ob.close()
     return dt, c1["seq_steps"] - c0["seq_steps"], c1["draft_tokens"] - c0["draft_tokens"], S
+
+
+def closed_loop(P, batch, seqs, spec, L):
+    """The whole decoding loop on the device: sam_step drafts, the sequences' own continuation plays
+    the target model, sam_accept_greedy verifies and produces the next step's input.  Reports the
+    mean number of accepted tokens per step (the paper's #MAT) and the time per loop iteration."""
+    import torch
+    B, total = seqs.shape
+    dev = batch.device
+    sd = P.binding
+    seq_dev = torch.from_numpy(seqs).to(dev).long()
+    stride = L + 1
+    nt = torch.empty((B, stride), dtype=torch.int32, device=dev)
+    cnt = torch.empty(B, dtype=torch.int32, device=dev)
+    acc = torch.empty_like(cnt)
+    ar = torch.arange(L + 1, device=dev)[None, :]
+    batch.reset()
+    out = batch.step(seq_dev[:, :spec.prompt_len].int().contiguous(),
+                     torch.full((B,), spec.prompt_len, dtype=torch.int32, device=dev), L)
+    pos = torch.full((B,), spec.prompt_len, dtype=torch.int64, device=dev)
+    steps = seq_steps = accepted_draft = 0
+    src_hist = torch.zeros(4, dtype=torch.int64, device=dev)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    while True:
+        target = torch.gather(seq_dev, 1, torch.clamp(pos[:, None] + ar, max=total - 1)).int().contiguous()
+        cap = (total - pos).int().contiguous()
+        sd.sam_accept_greedy(out.draft_tokens, out.draft_len, target, cap, nt, cnt, acc)
+        active = cnt > 0
+        src_hist += torch.bincount(out.source[active].long(), minlength=4)
+        seq_steps += int(active.sum().item())               # one host read per iteration, to know when to stop
+        accepted_draft += int(acc.sum().item())
+        if not bool(active.any().item()):
+            break
+        batch.step(nt, cnt, L, out)
+        pos += cnt.long()
+        steps += 1
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    gen = int((pos - spec.prompt_len).sum().item())
+    h = src_hist.tolist()
+    return {"decoding_steps": steps, "sequence_steps": seq_steps, "generated_tokens": gen,
+            "mean_accepted_tokens_per_step": gen / max(seq_steps, 1),
+            "mean_confirmed_draft_tokens_per_step": accepted_draft / max(seq_steps, 1),
+            "draft_source_share": {"none": h[0] / max(seq_steps, 1), "static": h[1] / max(seq_steps, 1),
+                                   "dynamic": h[2] / max(seq_steps, 1)},
+            "us_per_loop_iteration": dt * 1e6 / max(steps, 1),
+            "note": "target = the sequence's own continuation (synthetic); torch gathers the target rows"}
 
 
 def main_reference(args):
@@ -359,6 +409,9 @@ def main_ours(args):
         "clocks": clocks,
         "roofline": roofline,
     }
+
+    if args.closed_loop:
+        line["closed_loop"] = closed_loop(P, batch, seqs, spec, L)
 
     if world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
