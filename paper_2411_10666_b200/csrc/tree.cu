@@ -39,10 +39,10 @@ __device__ __forceinline__ int load_candidates(const SamStaticView& S, uint32_t 
     ordered = true;
     uint32_t at = sam_hash1(u) & S.topk_mask;
     for (uint32_t probe = 0; probe <= S.topk_mask; probe++) {
-        const uint4 h = __ldg(S.topk + (size_t)at * 4);
+        // the whole 64-byte entry in one round of reads; the header decides afterwards
+        const uint4 h = __ldg(S.topk + (size_t)at * 4), w1 = __ldg(S.topk + (size_t)at * 4 + 1),
+                    w2 = __ldg(S.topk + (size_t)at * 4 + 2), w3 = __ldg(S.topk + (size_t)at * 4 + 3);
         if (h.x == u) {
-            const uint4 w1 = __ldg(S.topk + (size_t)at * 4 + 1), w2 = __ldg(S.topk + (size_t)at * 4 + 2),
-                        w3 = __ldg(S.topk + (size_t)at * 4 + 3);
             // layout: {state, n, 0, 0} {tok0..3} {tok4, tok5, tgt0, tgt1} {tgt2..5}
             ctok[0] = w1.x; ctok[1] = w1.y; ctok[2] = w1.z; ctok[3] = w1.w; ctok[4] = w2.x; ctok[5] = w2.y;
             ctgt[0] = w2.z; ctgt[1] = w2.w; ctgt[2] = w3.x; ctgt[3] = w3.y; ctgt[4] = w3.z; ctgt[5] = w3.w;
