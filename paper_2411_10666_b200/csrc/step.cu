@@ -389,7 +389,13 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             if (D.err) return;
             D.n_states = cl + 1;
             uint4* rq = rec_ptr(D, q);
+            // the redirect walk's first read (the record of link[p]) does not depend on q's record:
+            // both go out together.  link[p] is neither p, q nor cl, so nothing below changes it.
+            const bool ahead = !at_root && lk.link != 0;
+            const uint4* rn = rec_ptr(D, ahead ? lk.link : q);
             const uint4 qa = rq[0], qb = rq[1];
+            uint4 na = make_uint4(0, 0, 0, 0), nb2 = make_uint4(0, 0, 0, 0);
+            if (ahead) { na = rn[0]; nb2 = rn[1]; }
             uint4 nb;
             if (qa.w <= 2) {
                 nb = make_uint4(qb.x, qb.y & SAM_IDMASK, qb.z, qb.w & SAM_IDMASK);   // copies are never solid
@@ -418,6 +424,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
                 }
                 uint32_t pp = lk.link;
                 int g2 = (int)plen + 2;
+                bool first = ahead;
                 for (;;) {
                     if (pp == 0) {
                         RootLook r2 = root_lookup(D, t);
@@ -425,7 +432,8 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
                         if (r2.found && (r2.tgt & SAM_IDMASK) == q) root_retarget(D, r2.slot, cl);
                         break;
                     }
-                    Look l2k = lookup_state(D, pp, t);
+                    Look l2k = lookup_state(D, pp, t, first, na, nb2);
+                    first = false;
                     if (!l2k.found) { D.err = SAM_SEQ_WALK_LIMIT; return; }   // every state up the chain has t
                     if ((l2k.tgt & SAM_IDMASK) != q) break;
                     uint32_t* rw2 = reinterpret_cast<uint32_t*>(rec_ptr(D, pp));
