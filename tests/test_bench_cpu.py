@@ -1,0 +1,58 @@
+"""Host-side checks of the benchmark and of the workload recipes (no GPU)."""
+import json
+import os
+import subprocess
+import sys
+
+import numpy as np
+
+import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_reference_arm_prints_one_json_line():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--steps", "40", "--warmup", "3"], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    j = json.loads(lines[0])
+    assert j["impl"] == "reference" and j["metric"] == "sam_sequence_steps_per_sec" and j["unit"] == "sequence-steps/s"
+    assert j["steps"] == 40 and j["warmup"] == 3 and j["value"] > 0 and j["higher_is_better"] is True
+    assert j["cpu_baseline"]["kind"] == "oracle" and j["cpu_baseline"]["cores"] >= 1
+    assert j["e2e"]["h2d_bytes_per_step"] == 0 and j["e2e"]["d2h_bytes_per_step"] == 0
+    assert j["config"]["workload"] == "tiny"
+
+
+def test_reference_arm_other_ranks_do_nothing():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--gpus", "2"], capture_output=True, text=True, timeout=120, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_recipes_have_the_stated_shape():
+    for name, spec in W.SPECS.items():
+        small = W.scaled(spec, corpus_len=min(spec.corpus_len, 200_000), batch=min(spec.batch, 8))
+        w = W.make(small)
+        assert w.corpus.shape == (small.corpus_len,) and w.corpus.dtype == np.int32
+        assert w.corpus.min() >= 0 and w.corpus.max() < spec.vocab
+        assert w.seqs.shape == (small.batch, spec.prompt_len + spec.gen_len)
+        assert w.seqs.min() >= 0 and w.seqs.max() < spec.vocab
+        c = w.counts
+        assert (c.sum(axis=0) == spec.gen_len).all() and c.max() <= spec.accept_max and c.min() >= 0
+        # the packed step rows are exactly the generated part, in order
+        for b in range(small.batch):
+            toks = np.concatenate([w.new_tokens[s, b, :c[s, b]] for s in range(w.n_steps)])
+            assert np.array_equal(toks, w.seqs[b, spec.prompt_len:])
+        assert (w.new_tokens[np.arange(spec.accept_max)[None, None, :] >= c[:, :, None]] == -1).all()
+        mean_m = c[c > 0].mean()
+        expect = {"tiny": 2.5, "c2": 2.46, "c3": 2.77, "c4": 3.87, "c5": 3.32}[name]
+        assert abs(mean_m - expect) < 0.35, (name, mean_m)
+    # seeds: same recipe twice gives the same arrays; another seed differs
+    a = W.make(W.scaled(W.SPECS["tiny"], corpus_len=5000))
+    b = W.make(W.scaled(W.SPECS["tiny"], corpus_len=5000))
+    c2 = W.make(W.scaled(W.SPECS["tiny"], corpus_len=5000, seed=7))
+    assert np.array_equal(a.corpus, b.corpus) and np.array_equal(a.seqs, b.seqs)
+    assert not np.array_equal(a.corpus, c2.corpus)
