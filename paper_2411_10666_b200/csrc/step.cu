@@ -80,10 +80,11 @@ __device__ __forceinline__ int cut_at_stop(int32_t d[MAX_DRAFT_REGS], int dl, in
 
 // ------------------------------------------------------------------ static side
 // Transfer (Algorithm 1) for one token.  (s, sf, l): state, its F bit, match length.
-// root_e is root_row[t], fetched beforehand.  If have_rec, (pa, pb) is the record of s, read earlier.
+// root_e is root_row[t], fetched beforehand.  If have_rec, (pa, pb) is the record of s, read earlier;
+// if have_ent, pent is this lane's entry of the home bucket of (s, t), read earlier.
 __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t& s, uint32_t& sf, int32_t& l,
                                                 uint32_t t, uint32_t root_e, int lane, int& err,
-                                                bool have_rec, uint4 pa, uint4 pb) {
+                                                bool have_rec, uint4 pa, uint4 pb, bool have_ent, uint4 pent) {
     int guard = l + 2;                       // at most l link moves
     bool len_from_rec = false;
     for (;;) {
@@ -94,7 +95,8 @@ __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t
         }
         uint32_t home = sam_hash2(s, t) & S.hash_mask;
         uint4 ent = make_uint4(SAM_NONE, 0, 0, 0);
-        if (sf) ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+        if (sf) ent = have_ent ? pent : __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+        have_ent = false;
         uint4 a = pa, b = pb;
         if (!have_rec) { a = __ldg(S.rec + 2 * (size_t)s); b = __ldg(S.rec + 2 * (size_t)s + 1); }
         have_rec = false;
@@ -584,9 +586,48 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                 uint32_t tk = 0, re = SAM_NONE;
                 if (i < m) { tk = (uint32_t)(base == 0 ? tok_first : toks[i]); re = __ldg(A.S.root_row + tk); }
                 const int cnt = min(32, m - base);
+                // Most tokens end a short match: the lookup misses, the link leads to the root, and the
+                // root row gives the next state u = root_row[t].  The token after that is then looked up
+                // in u — a lookup whose address is known now.  Lookups k = 0..7 (state root_row[t_k],
+                // token t_{k+1}) are read ahead here, eight lanes each: the state's record in lanes 0-1
+                // of the group, its hash bucket in all eight.  They are used if the matcher really is
+                // in that state when the token comes.
+                uint4 sp_rec[2], sp_ent[2];
+#pragma unroll
+                for (int r = 0; r < 2; r++) {
+                    const int k = 4 * r + (lane >> 3), e = lane & 7;
+                    const uint32_t uref = __shfl_sync(FULL, re, k);
+                    const uint32_t tnext = __shfl_sync(FULL, tk, k + 1);
+                    sp_rec[r] = make_uint4(0, 0, 0, 0);
+                    sp_ent[r] = make_uint4(SAM_NONE, 0, 0, 0);
+                    if (k + 1 < cnt && uref != SAM_NONE) {
+                        const uint32_t u = uref & SAM_IDMASK;
+                        if (e < 2) sp_rec[r] = __ldg(A.S.rec + 2 * (size_t)u + e);
+                        if (uref >> 31)
+                            sp_ent[r] = __ldg(A.S.hash + (size_t)(sam_hash2(u, tnext) & A.S.hash_mask) * SAM_HASH_BUCKET + e);
+                    }
+                }
                 for (int j = 0; j < cnt && !err; j++) {
+                    bool pre = false;
+                    uint4 pa = ra, pb = rb, pent = make_uint4(SAM_NONE, 0, 0, 0);
+                    if (j >= 1 && j <= 8 && s != 0) {
+                        const uint32_t prev = __shfl_sync(FULL, re, j - 1);
+                        if (prev != SAM_NONE && (prev & SAM_IDMASK) == s) {        // the state read ahead
+                            const int k = j - 1, g8 = 8 * (k & 3);
+                            const uint4 xr = (k >> 2) ? sp_rec[1] : sp_rec[0];
+                            const uint4 xe = (k >> 2) ? sp_ent[1] : sp_ent[0];
+                            pa.x = __shfl_sync(FULL, xr.x, g8); pa.y = __shfl_sync(FULL, xr.y, g8);
+                            pa.z = __shfl_sync(FULL, xr.z, g8); pa.w = __shfl_sync(FULL, xr.w, g8);
+                            pb.x = __shfl_sync(FULL, xr.x, g8 + 1); pb.y = __shfl_sync(FULL, xr.y, g8 + 1);
+                            pb.z = __shfl_sync(FULL, xr.z, g8 + 1); pb.w = __shfl_sync(FULL, xr.w, g8 + 1);
+                            const int src = g8 + (lane & 7);
+                            pent.x = __shfl_sync(FULL, xe.x, src); pent.y = __shfl_sync(FULL, xe.y, src);
+                            pent.z = __shfl_sync(FULL, xe.z, src); pent.w = __shfl_sync(FULL, xe.w, src);
+                            pre = true;
+                        }
+                    }
                     static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err,
-                                    have, ra, rb);
+                                    have || pre, pa, pb, pre, pent);
                     have = false;
                 }
             }
