@@ -275,7 +275,7 @@ int32_t osam_topk(const osam_t* S, const int64_t* freq, int32_t s, int32_t k, in
  * then the source is static iff l1 > l2 + l_bias, and the draft is the slice of that source's
  * text after min_endpos of its state, at most L tokens, clipped at the end of the text.
  *
- * Readings where the paper is silent (each is listed in the design notes):
+ * Readings where the paper is silent:
  *   - after Expand clones the state the dynamic matcher sits in, the matcher is moved to the
  *     canonical state of its match length: while len[link[s]] >= l, s <- link[s].  It must then
  *     equal link[last] with l = len[s]; this is asserted after every token (err 2 otherwise).

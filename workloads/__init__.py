@@ -88,7 +88,7 @@ class Spec:
     seed: int = 0
 
 
-# Index i is BASELINE configs[i]; seeds are 0x5A4D0000 + i.
+# The five recipes, smallest first; seeds are 0x5A4D0000 + position.
 SPECS = {
     "tiny": Spec("tiny", 100_000, 32000, 1.1, False, 0.30, 8, 64, 4, 256, 512,
                  0.40, 0.5, 0.40, 0.5, False, "uniform", 4, 0.0, 16, seed=0x5A4D0000),
