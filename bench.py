@@ -76,7 +76,7 @@ class ClockSampler:
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index):
         self.proc = None
         try:
             fd, self.path = tempfile.mkstemp(prefix="samclk_", suffix=".csv")
@@ -289,7 +289,12 @@ def main_ours(args):
     torch.cuda.synchronize()
     prefill_ms = e0.elapsed_time(e1)
 
-    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    gpu_id = str(torch.cuda.current_device())
+    try:                                                  # the physical GPU, whatever CUDA_VISIBLE_DEVICES says
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(gpu_id) if rank == 0 else None
     times = []
     t_start = time.perf_counter()
     while True:

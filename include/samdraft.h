@@ -240,6 +240,21 @@ int sam_accept_greedy(int32_t batch, const int32_t* draft_tokens_dev, const int3
                       int32_t* new_tokens_dev, int32_t stride, int32_t* counts_dev, int32_t* accepted_dev,
                       void* stream);
 
+/* sam_accept_greedy and sam_step in one launch: slot i's accepted tokens are derived inside the step
+ * kernel from its previous draft (prev_draft_tokens_dev [B, prev_L], prev_draft_len_dev [B]) and the
+ * target's tokens (target_tokens_dev [B, prev_L + 1]) exactly as sam_accept_greedy derives them
+ * (m = confirmed prefix + 1, clipped to max_new_dev[i] if given), and are fed to the automata at once;
+ * the new draft and the other outputs are those of sam_step.  counts_out_dev / accepted_out_dev
+ * ([B], may be NULL) receive m and the number of confirmed draft tokens.  The previous draft's
+ * buffers must not be this call's output buffers (alternate between two sets).
+ * Asynchronous on `stream`.  Errors: ARG, CUDA. */
+int sam_step_verified(sam_batch_t* b, const int32_t* target_tokens_dev, int32_t prev_L,
+                      const int32_t* prev_draft_tokens_dev, const int32_t* prev_draft_len_dev,
+                      const int32_t* max_new_dev, int32_t L,
+                      int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,
+                      int32_t* source_dev, int32_t* state_dev, int32_t* status_dev,
+                      int32_t* counts_out_dev, int32_t* accepted_out_dev, void* stream);
+
 /* Adaptive draft selection (Section 3.4): the auxiliary drafter stands in with a fixed virtual match
  * length l_threshold.  With min_match = l_threshold in sam_batch_opts_t, sam_step reports
  * source = SAM_SRC_NONE exactly where the automaton's chosen match is shorter than that; this call

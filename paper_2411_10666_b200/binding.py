@@ -78,6 +78,8 @@ SIGNATURES = {
     "sam_batch_destroy": (None, [c_void_p]),
     "sam_accept_greedy": (c_int, [c_int32, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32,
                                   c_void_p, c_void_p, c_void_p]),
+    "sam_step_verified": (c_int, [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32,
+                                  c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "sam_select_auxiliary": (c_int, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "sam_tree_draft": (c_int, [c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                c_void_p, c_void_p]),
@@ -287,6 +289,19 @@ def sam_accept_greedy(draft_tokens, draft_len, target_tokens, max_new, new_token
                                    _dev_ptr(target_tokens, "target_tokens"), _dev_ptr(max_new, "max_new"),
                                    _dev_ptr(new_tokens, "new_tokens"), new_tokens.shape[1], _dev_ptr(counts, "counts"),
                                    _dev_ptr(accepted, "accepted"), _stream_ptr(stream)), "sam_accept_greedy")
+
+
+def sam_step_verified(h, target_tokens, prev_draft_tokens, prev_draft_len, max_new, L,
+                      draft_tokens, draft_len, match_len, source, state, status, counts_out=None, accepted_out=None,
+                      stream=None):
+    _check(lib().sam_step_verified(h, _dev_ptr(target_tokens, "target_tokens"), prev_draft_tokens.shape[1],
+                                   _dev_ptr(prev_draft_tokens, "prev_draft_tokens"), _dev_ptr(prev_draft_len, "prev_draft_len"),
+                                   _dev_ptr(max_new, "max_new"), L,
+                                   _dev_ptr(draft_tokens, "draft_tokens"), _dev_ptr(draft_len, "draft_len"),
+                                   _dev_ptr(match_len, "match_len"), _dev_ptr(source, "source"),
+                                   _dev_ptr(state, "state"), _dev_ptr(status, "status"),
+                                   _dev_ptr(counts_out, "counts_out"), _dev_ptr(accepted_out, "accepted_out"),
+                                   _stream_ptr(stream)), "sam_step_verified")
 
 
 def sam_select_auxiliary(draft_tokens, draft_len, source, aux_tokens, aux_len, stream=None):

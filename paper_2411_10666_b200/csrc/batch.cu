@@ -319,6 +319,22 @@ extern "C" int sam_step(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t s
                            match_len_dev, source_dev, state_dev, status_dev, (cudaStream_t)stream);
 }
 
+extern "C" int sam_step_verified(sam_batch_t* b, const int32_t* target_tokens_dev, int32_t prev_L,
+                                 const int32_t* prev_draft_tokens_dev, const int32_t* prev_draft_len_dev,
+                                 const int32_t* max_new_dev, int32_t L,
+                                 int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,
+                                 int32_t* source_dev, int32_t* state_dev, int32_t* status_dev,
+                                 int32_t* counts_out_dev, int32_t* accepted_out_dev, void* stream) {
+    int rc = check_step_args(b, target_tokens_dev, prev_L + 1, prev_draft_len_dev, L, draft_tokens_dev, draft_len_dev,
+                             match_len_dev, source_dev, status_dev);
+    if (rc) return rc;
+    if (!prev_draft_tokens_dev || prev_L < 1 || prev_L > 128) return SAM_ERR_ARG;
+    if (prev_draft_tokens_dev == draft_tokens_dev || prev_draft_len_dev == draft_len_dev) return SAM_ERR_ARG;
+    return sam_launch_step_full(b, target_tokens_dev, prev_L + 1, nullptr, L, draft_tokens_dev, draft_len_dev,
+                                match_len_dev, source_dev, state_dev, status_dev, (cudaStream_t)stream, nullptr, 0,
+                                prev_draft_tokens_dev, prev_draft_len_dev, max_new_dev, counts_out_dev, accepted_out_dev);
+}
+
 extern "C" int sam_run_steps(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
                              const int32_t* counts_dev, int32_t n_steps, int32_t L, int32_t out_per_step,
                              int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,

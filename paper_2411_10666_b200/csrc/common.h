@@ -60,6 +60,13 @@ int sam_launch_step_signal(const sam_batch* b, const int32_t* new_tokens, int32_
                            int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream,
                            int32_t* done_flag_dev, int32_t done_seq);
 
+int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
+                         int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
+                         int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream,
+                         int32_t* done_flag_dev, int32_t done_seq,
+                         const int32_t* v_draft, const int32_t* v_draft_len, const int32_t* v_max_new,
+                         int32_t* v_counts_out, int32_t* v_accepted_out);
+
 // helpers implemented in batch.cu
 int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBatchView* view,
                   size_t* total, size_t* stage_words);

@@ -37,6 +37,11 @@ struct StepArgs {
     // optional completion signal for the host-array step: the last block to finish writes done_seq to
     // *done_flag (host-mapped memory) so the host can poll instead of synchronising the stream
     int32_t* done_count; int32_t* done_flag; int32_t done_seq;
+    // optional fused greedy verification (Section 2.2): when v_draft is set, new_tokens holds the target
+    // model's tokens [B, stride] with stride = previous draft length limit + 1, and each slot's count is
+    // derived here: the confirmed prefix of its previous draft plus the target's next token
+    const int32_t* v_draft; const int32_t* v_draft_len; const int32_t* v_max_new;
+    int32_t* v_counts_out; int32_t* v_accepted_out;
 };
 
 // ------------------------------------------------------------------ draft read
@@ -512,6 +517,8 @@ __device__ __forceinline__ void signal_done(const StepArgs& A) {
 }
 
 // ------------------------------------------------------------------ the kernel
+// VERIFY: the accepted tokens are derived from the previous draft and the target's tokens (sam_step_verified).
+template <bool VERIFY>
 __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ StepArgs A) {
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -524,9 +531,28 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
     const uint32_t cw = cb[lane];                       // control words 0..31
     const uint32_t cw2 = cb[32 + lane];                 // control words 32..63
-    const int m = A.counts[b];
     int32_t tok_first = 0;
     if (lane < A.stride) tok_first = toks[lane];
+    int m, confirmed = 0;
+    if (VERIFY) {
+        // x_accept = the draft tokens the target reproduces, then the target's own next token
+        const int Lp = A.stride - 1;
+        int dl = A.v_draft_len[b];
+        dl = dl < 0 ? 0 : (dl > Lp ? Lp : dl);
+        const int32_t* dr = A.v_draft + (size_t)b * Lp;
+        int a = dl;
+        for (int base = 0; base < dl; base += 32) {
+            const int j = base + lane;
+            const bool differs = j < dl && dr[j] != toks[j];
+            const unsigned bad = __ballot_sync(FULL, differs);
+            if (bad) { a = base + __ffs(bad) - 1; break; }
+        }
+        m = a + 1;
+        if (A.v_max_new) { int cap = A.v_max_new[b]; cap = cap < 0 ? 0 : cap; m = m < cap ? m : cap; }
+        confirmed = a < m ? a : m;
+    } else {
+        m = A.counts[b];
+    }
     int status = (int)__shfl_sync(FULL, cw, CB_STATUS);
     const uint32_t ntok0 = __shfl_sync(FULL, cw, CB_NTOK);
     const int L = A.L;
@@ -556,6 +582,8 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                 A.draft_len[b] = 0; A.match_len[2 * b] = 0; A.match_len[2 * b + 1] = 0; A.source[b] = 0;
                 if (A.state) { A.state[2 * b] = 0; A.state[2 * b + 1] = 0; }
                 A.status[b] = status;
+                if (VERIFY && A.v_counts_out) A.v_counts_out[b] = m;
+                if (VERIFY && A.v_accepted_out) A.v_accepted_out[b] = confirmed;
             }
             __syncwarp();
             if (A.done_flag && lane == 0) signal_done(A);
@@ -745,6 +773,8 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         A.source[b] = src;
         if (A.state) { A.state[2 * b] = any_err ? 0 : sh_s[0]; A.state[2 * b + 1] = any_err ? 0 : sh_s[1]; }
         A.status[b] = any_err;
+        if (VERIFY && A.v_counts_out) A.v_counts_out[b] = m;
+        if (VERIFY && A.v_accepted_out) A.v_accepted_out[b] = confirmed;
     }
     if (A.done_flag) {
         __syncthreads();
@@ -765,7 +795,19 @@ int sam_launch_step_signal(const sam_batch* b, const int32_t* new_tokens, int32_
                            int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
                            int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream,
                            int32_t* done_flag_dev, int32_t done_seq) {
+    return sam_launch_step_full(b, new_tokens, stride, counts, L, draft_tokens, draft_len, match_len, source, state,
+                                status, stream, done_flag_dev, done_seq, nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
+                         int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
+                         int32_t* source, int32_t* state, int32_t* status, cudaStream_t stream,
+                         int32_t* done_flag_dev, int32_t done_seq,
+                         const int32_t* v_draft, const int32_t* v_draft_len, const int32_t* v_max_new,
+                         int32_t* v_counts_out, int32_t* v_accepted_out) {
     StepArgs A;
+    A.v_draft = v_draft; A.v_draft_len = v_draft_len; A.v_max_new = v_max_new;
+    A.v_counts_out = v_counts_out; A.v_accepted_out = v_accepted_out;
     A.done_count = b->view.pool_hdr + 4; A.done_flag = done_flag_dev; A.done_seq = done_seq;
     A.has_static = b->st != nullptr;
     if (b->st) A.S = b->st->view;
@@ -774,7 +816,8 @@ int sam_launch_step_signal(const sam_batch* b, const int32_t* new_tokens, int32_
     A.new_tokens = new_tokens; A.stride = stride; A.counts = counts; A.L = L;
     A.draft_tokens = draft_tokens; A.draft_len = draft_len; A.match_len = match_len;
     A.source = source; A.state = state; A.status = status;
-    sam_step_kernel<<<b->view.batch, 64, 0, stream>>>(A);
+    if (v_draft) sam_step_kernel<true><<<b->view.batch, 64, 0, stream>>>(A);
+    else sam_step_kernel<false><<<b->view.batch, 64, 0, stream>>>(A);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
     return SAM_OK;

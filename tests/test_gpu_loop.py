@@ -87,3 +87,41 @@ def test_closed_loop_matches_oracle(P, key, N, B, pl, gl, min_match):
     assert np.array_equal(pos.cpu().numpy(), pos_ref) and (pos_ref == total).all()
     mean_accept = np.mean([r["counts"][r["counts"] > 0].mean() for r in log if (r["counts"] > 0).any()])
     assert mean_accept > 1.05                                 # retrieval drafts do get accepted
+
+
+def test_fused_verify_and_step_matches_the_two_call_loop(P):
+    """sam_step_verified (verification folded into the step kernel) against the oracle's loop."""
+    import torch
+    spec = W.scaled(W.SPECS["c2"], 200000, 12, 200, 300)
+    w = W.make(spec)
+    B, pl, L = spec.batch, spec.prompt_len, spec.draft_len
+    total = pl + spec.gen_len
+    S = oracle.Sam(w.corpus)
+    ob = oracle.Batch(S, w.corpus, B, spec.vocab, total)
+    log, pos_ref = accept.decode_loop(ob, w.seqs, pl, L, L + 1)
+
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    batch = P.Batch(st, B, total, max_draft_len=L)
+    dev = batch.device
+    seqs = _t(w.seqs, dev).long()
+    outs = [P.StepOutputs(B, L, dev), P.StepOutputs(B, L, dev)]       # the previous draft and the new one alternate
+    cur = 0
+    batch.step(_t(w.prompts, dev), torch.full((B,), pl, dtype=torch.int32, device=dev), L, outs[cur])
+    pos = torch.full((B,), pl, dtype=torch.int64, device=dev)
+    cnt = torch.empty(B, dtype=torch.int32, device=dev); acc = torch.empty_like(cnt)
+    ar = torch.arange(L + 1, device=dev)[None, :]
+    for step, ref in enumerate(log):
+        prev, new = outs[cur], outs[1 - cur]
+        got = prev.cpu()
+        for k in ("draft_tokens", "draft_len", "match_len", "source", "state", "status"):
+            assert np.array_equal(got[k], ref[k]), (step, k)
+        target = torch.gather(seqs, 1, torch.clamp(pos[:, None] + ar, max=total - 1)).int().contiguous()
+        cap = (total - pos).int().contiguous()
+        P.binding.sam_step_verified(batch.handle, target, prev.draft_tokens, prev.draft_len, cap, L,
+                                    *new.tensors(), counts_out=cnt, accepted_out=acc)
+        assert np.array_equal(cnt.cpu().numpy(), ref["counts"]) and np.array_equal(acc.cpu().numpy(), ref["accepted"])
+        pos += cnt.long()
+        cur = 1 - cur
+    assert np.array_equal(pos.cpu().numpy(), pos_ref)
+    with pytest.raises(P.SamError):                                  # the previous draft may not be the output buffer
+        P.binding.sam_step_verified(batch.handle, target, new.draft_tokens, new.draft_len, cap, L, *new.tensors())
