@@ -60,6 +60,8 @@ def parse_args():
     ap.add_argument("--max-repeats", type=int, default=300)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probes", action="store_true")
+    ap.add_argument("--tree-draft", action="store_true",
+                    help="also time sam_tree_draft (builds the static automaton with top-k successor data)")
     ap.add_argument("--closed-loop", action="store_true",
                     help="also run draft -> verify -> accept -> update on the device with the true continuation as target")
     return ap.parse_args()
@@ -161,6 +163,36 @@ def run_oracle_timed(spec, corpus, seqs, counts, new_tokens, steps_lo, steps_hi,
     return dt, c1["seq_steps"] - c0["seq_steps"], c1["draft_tokens"] - c0["draft_tokens"], S
 
 
+def tree_draft_timing(P, st, batch, prepare, out, flush):
+    """Time sam_tree_draft (best-first tree over the top-k successors, Algorithm 5) from the static states
+    the batch is in after the warm-up steps; L2 flushed before every call."""
+    import torch
+    prepare()
+    torch.cuda.synchronize()
+    B = batch.batch
+    dev = batch.device
+    states = out.state[:, 0].contiguous()
+    starts = torch.zeros(B, dtype=torch.int32, device=dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    res = {"slots_with_a_static_match": int((states > 0).sum().item())}
+    for max_size, k in ((16, 2), (40, 4), (70, 4)):
+        toks = torch.empty((B, max_size), dtype=torch.int32, device=dev)
+        par = torch.empty_like(toks)
+        sz = torch.empty(B, dtype=torch.int32, device=dev)
+        ts = []
+        for _ in range(15):
+            flush.zero_()
+            torch.cuda.synchronize()
+            e0.record()
+            P.binding.sam_tree_draft(st.handle, states, starts, max_size, k, toks, par, None, sz)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        res["max_size_%d_k_%d" % (max_size, k)] = {"us_per_call": statistics.median(ts),
+                                                   "mean_tree_size": float(sz.float().mean().item())}
+    return res
+
+
 def closed_loop(P, batch, seqs, spec, L):
     """The whole decoding loop on the device: sam_step drafts, the sequences' own continuation plays
     the target model, sam_accept_greedy verifies and produces the next step's input.  Reports the
@@ -259,7 +291,7 @@ def main_ours(args):
     assert K >= 1 and Wm >= 3, "need at least 3 warm-up steps and 1 timed step"
 
     t0 = time.perf_counter()
-    st = P.StaticSam.build(corpus, spec.vocab, device=local_rank)
+    st = P.StaticSam.build(corpus, spec.vocab, device=local_rank, tree_topk=4 if args.tree_draft else 0)
     build_s = time.perf_counter() - t0
     info = st.info
     batch = P.Batch(st, B, msl, max_draft_len=L, max_host_stride=spec.accept_max)
@@ -444,6 +476,8 @@ def main_ours(args):
         "roofline": roofline,
     }
 
+    if args.tree_draft:
+        line["tree_draft"] = tree_draft_timing(P, st, batch, prepare, out, flush)
     if args.closed_loop:
         line["closed_loop"] = closed_loop(P, batch, seqs, spec, L)
 
