@@ -22,6 +22,8 @@
 //     in parallel (each such Expand is three independent writes).
 #include "common.h"
 
+#include <cstring>
+
 namespace {
 
 constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -520,6 +522,11 @@ __device__ __forceinline__ void signal_done(const StepArgs& A) {
 // VERIFY: the accepted tokens are derived from the previous draft and the target's tokens (sam_step_verified).
 template <bool VERIFY>
 __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ StepArgs A) {
+    // Programmatic dependent launch: this grid may be scheduled while the previous kernel of the stream
+    // is still finishing.  Nothing is read before that kernel has completed and flushed; the kernel
+    // after this one is allowed to get scheduled right away (it waits in the same way).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __shared__ int32_t sh_l[2], sh_s[2], sh_dl[2], sh_err[2];
@@ -816,9 +823,16 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
     A.new_tokens = new_tokens; A.stride = stride; A.counts = counts; A.L = L;
     A.draft_tokens = draft_tokens; A.draft_len = draft_len; A.match_len = match_len;
     A.source = source; A.state = state; A.status = status;
-    if (v_draft) sam_step_kernel<true><<<b->view.batch, 64, 0, stream>>>(A);
-    else sam_step_kernel<false><<<b->view.batch, 64, 0, stream>>>(A);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)b->view.batch); cfg.blockDim = dim3(64); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaError_t e = v_draft ? cudaLaunchKernelEx(&cfg, sam_step_kernel<true>, A)
+                            : cudaLaunchKernelEx(&cfg, sam_step_kernel<false>, A);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
     return SAM_OK;
 }
