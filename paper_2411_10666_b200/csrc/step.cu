@@ -211,17 +211,25 @@ __device__ __forceinline__ Look lookup_state(const Dyn& D, uint32_t p, uint32_t 
         else if (a.w == 2 && b.z == t) { r.found = true; r.tgt = b.w; r.idx = 1; }
         return r;
     }
+    // 128 entries per round trip: the four reads of a lane are independent and go out together
     const uint2* blk = blk_ptr(D, b.x);
-    for (uint32_t base = 0; base < a.w; base += 32) {
-        uint32_t i = base + D.lane;
-        uint2 e = make_uint2(SAM_NONE, 0);
-        if (i < a.w) e = blk[i];
-        unsigned hit = __ballot_sync(FULL, e.x == t);
-        if (hit) {
-            int src = __ffs(hit) - 1;
-            r.found = true; r.tgt = __shfl_sync(FULL, e.y, src); r.idx = base + src;
-            break;
+    for (uint32_t base = 0; base < a.w; base += 128) {
+        uint2 e[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const uint32_t i = base + 32 * u + D.lane;
+            e[u] = make_uint2(SAM_NONE, 0);
+            if (i < a.w) e[u] = blk[i];
         }
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const unsigned hit = __ballot_sync(FULL, e[u].x == t);
+            if (hit && !r.found) {
+                const int src = __ffs(hit) - 1;
+                r.found = true; r.tgt = __shfl_sync(FULL, e[u].y, src); r.idx = base + 32 * u + src;
+            }
+        }
+        if (r.found) break;
     }
     return r;
 }
