@@ -13,7 +13,7 @@ constexpr size_t SAM_ZERO_COPY_MAX_BYTES = 256u << 10;   // larger host steps go
 constexpr int SAM_POLL_LIMIT_US = 2000;                  // how long a host step polls its completion flag
 
 struct WsLayout {
-    size_t off_hdr, off_ctrl, off_free, off_owner, off_reset, off_text, off_root, off_stage, off_pool, total;
+    size_t off_hdr, off_ctrl, off_free, off_owner, off_reset, off_text, off_pstate, off_root, off_stage, off_pool, total;
     int32_t text_stride, root_cap, slab_shift, pool_slabs, max_host_stride;
     size_t stage_words;
 };
@@ -53,6 +53,7 @@ int plan(const sam_batch_opts_t* o, WsLayout* w) {
     w->off_owner = off; off = sam_align_up(off + (size_t)slabs * 4, 256);
     w->off_reset = off; off = sam_align_up(off + (size_t)o->batch * 4 * 2, 256);   // flags + slot list
     w->off_text = off;  off = sam_align_up(off + (size_t)o->batch * w->text_stride * 4, 256);
+    w->off_pstate = off; off = sam_align_up(off + (size_t)o->batch * w->text_stride * 4, 256);
     w->off_root = off;  off = sam_align_up(off + (size_t)o->batch * w->root_cap * 8, 256);
     w->off_stage = off; off = sam_align_up(off + w->stage_words * 4, 256);
     w->off_pool = off;  off = sam_align_up(off + (size_t)slabs * slab, 256);
@@ -173,6 +174,7 @@ int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBa
         view->slab_owner = (int32_t*)(b + w.off_owner);
         view->reset_flag = (int32_t*)(b + w.off_reset);
         view->text = (int32_t*)(b + w.off_text);
+        view->pstate = (uint32_t*)(b + w.off_pstate);
         view->root_tab = (uint2*)(b + w.off_root);
         view->stage = (int32_t*)(b + w.off_stage);
         view->pool = (unsigned char*)(b + w.off_pool);
@@ -239,6 +241,7 @@ extern "C" int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* 
     V.slab_owner = (int32_t*)(base + w.off_owner);
     V.reset_flag = (int32_t*)(base + w.off_reset);
     V.text = (int32_t*)(base + w.off_text);
+    V.pstate = (uint32_t*)(base + w.off_pstate);
     V.root_tab = (uint2*)(base + w.off_root);
     V.stage = (int32_t*)(base + w.off_stage);
     V.pool = (unsigned char*)(base + w.off_pool);

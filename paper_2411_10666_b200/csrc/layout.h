@@ -31,6 +31,9 @@
 //               32 consecutive entries per probe; a single lane can settle most lookups from the
 //               home bucket alone (found, or absent because the bucket still has an empty entry).
 //   text      : per slot, int32[max_seq_len].
+//   pstate    : per slot, uint32[max_seq_len]: pstate[i] is the id of the state Expand created for token i
+//               (the state of the whole prefix of length i + 1), so the states along an earlier
+//               occurrence of a passage can be addressed without following their transitions.
 #pragma once
 #include <stdint.h>
 #include <vector_types.h>
@@ -114,6 +117,7 @@ struct SamBatchView {
     int32_t* slab_owner;      // [pool_slabs], -1 = free
     int32_t* reset_flag;      // [B]
     int32_t* text;            // [B][text_stride]
+    uint32_t* pstate;         // [B][text_stride]: id of the state created by each text position
     uint2* root_tab;          // [B][root_cap]
     unsigned char* pool;      // pool_slabs * slab_bytes
     int32_t* stage;           // staging for sam_step_host (inputs then outputs)

@@ -134,6 +134,7 @@ struct Dyn {
     unsigned char* pool;
     uint2* root;                 // this slot's root table
     int32_t* text;               // this slot's token text
+    uint32_t* pstate;            // this slot's position -> state map (the state each token created)
     int32_t* pool_hdr; int32_t* free_stack; int32_t* slab_owner;
     uint32_t* cb;                // this slot's control block
     uint32_t tab;                // lane i: slab index of state slab i
@@ -143,6 +144,12 @@ struct Dyn {
     // (root_precompute): pr_state 0 = not known (or stale), 1 = present, 2 = absent.
     uint32_t pr_state, pr_tgt, pr_slot, pr_bucket;
     int cur;                     // lane that holds the answer for the token being processed
+};
+
+struct Pre {                     // records read ahead for the clone branch of Expand, kept in shared memory
+    bool valid;
+    uint32_t q;                  // rec[0..1] is the record of q, rec[2..3] that of link[s2] (if it is not the root)
+    const uint4* rec;
 };
 
 struct Look {                    // result of looking a token up in a non-root state
@@ -340,12 +347,39 @@ __device__ __forceinline__ void root_retarget(Dyn& D, uint32_t slot, uint32_t tg
     if (D.pr_state == 1 && D.pr_slot == slot) D.pr_tgt = tgt;
 }
 
+// The redirect loop of Expand's clone branch (Algorithm 3): from state pp up the suffix links, every
+// t-transition that leads to q is pointed to the clone cl instead; the walk ends at the first state
+// whose t-transition leads elsewhere, or past the root.  If first, (na, nb2) is the record of pp.
+__device__ __forceinline__ void redirect_walk(Dyn& D, uint32_t pp, uint32_t t, uint32_t q, uint32_t cl, int guard,
+                                              bool first, uint4 na, uint4 nb2) {
+    for (;;) {
+        if (pp == 0) {
+            RootLook r2 = root_lookup(D, t);
+            if (D.err) return;
+            if (r2.found && (r2.tgt & SAM_IDMASK) == q) root_retarget(D, r2.slot, cl);
+            return;
+        }
+        Look l2k = lookup_state(D, pp, t, first, na, nb2);
+        first = false;
+        if (!l2k.found) { D.err = SAM_SEQ_WALK_LIMIT; return; }   // every state up the chain has t
+        if ((l2k.tgt & SAM_IDMASK) != q) return;
+        uint32_t* rw2 = reinterpret_cast<uint32_t*>(rec_ptr(D, pp));
+        if (D.lane == 0) {
+            if (l2k.deg <= 2) rw2[5 + 2 * l2k.idx] = cl;
+            else blk_ptr(D, l2k.b0)[l2k.idx].y = cl;
+        }
+        pp = l2k.link;
+        if (--guard < 0) { D.err = SAM_SEQ_WALK_LIMIT; return; }
+    }
+}
+
 // Expand (Algorithm 3) for token t, fused with the dynamic matcher's Transfer.
 // last: state of the whole text; ntok: text length; (s2, l2): match state = link[last], its length.
 // On entry, if have_rec, (pa, pb) is the record of s2 as it stands; on exit have_rec says whether
 // (pa, pb) is the record of the new s2 (known without a read when s2 is a fresh clone).
 __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, uint32_t& ntok,
-                                           uint32_t& s2, uint32_t& l2, bool& have_rec, uint4& pa, uint4& pb) {
+                                           uint32_t& s2, uint32_t& l2, bool& have_rec, uint4& pa, uint4& pb,
+                                           const Pre& pre) {
     bool use_rec = have_rec;
     have_rec = false;
     const uint32_t k = ntok + 1;                       // max_length after this token
@@ -410,9 +444,14 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             // both go out together.  link[p] is neither p, q nor cl, so nothing below changes it.
             const bool ahead = !at_root && lk.link != 0;
             const uint4* rn = rec_ptr(D, ahead ? lk.link : q);
-            const uint4 qa = rq[0], qb = rq[1];
-            uint4 na = make_uint4(0, 0, 0, 0), nb2 = make_uint4(0, 0, 0, 0);
-            if (ahead) { na = rn[0]; nb2 = rn[1]; }
+            uint4 qa, qb, na = make_uint4(0, 0, 0, 0), nb2 = make_uint4(0, 0, 0, 0);
+            if (pre.valid && pre.q == q) {              // both were read by a run attempt that did not apply
+                qa = pre.rec[0]; qb = pre.rec[1];
+                if (ahead) { na = pre.rec[2]; nb2 = pre.rec[3]; }
+            } else {
+                qa = rq[0]; qb = rq[1];
+                if (ahead) { na = rn[0]; nb2 = rn[1]; }
+            }
             uint4 nb;
             if (qa.w <= 2) {
                 nb = make_uint4(qb.x, qb.y & SAM_IDMASK, qb.z, qb.w & SAM_IDMASK);   // copies are never solid
@@ -439,28 +478,8 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
                     if (lk.deg <= 2) rw[5 + 2 * lk.idx] = cl | SAM_FLAG;
                     else blk_ptr(D, lk.b0)[lk.idx].y = cl | SAM_FLAG;
                 }
-                uint32_t pp = lk.link;
-                int g2 = (int)plen + 2;
-                bool first = ahead;
-                for (;;) {
-                    if (pp == 0) {
-                        RootLook r2 = root_lookup(D, t);
-                        if (D.err) return;
-                        if (r2.found && (r2.tgt & SAM_IDMASK) == q) root_retarget(D, r2.slot, cl);
-                        break;
-                    }
-                    Look l2k = lookup_state(D, pp, t, first, na, nb2);
-                    first = false;
-                    if (!l2k.found) { D.err = SAM_SEQ_WALK_LIMIT; return; }   // every state up the chain has t
-                    if ((l2k.tgt & SAM_IDMASK) != q) break;
-                    uint32_t* rw2 = reinterpret_cast<uint32_t*>(rec_ptr(D, pp));
-                    if (D.lane == 0) {
-                        if (l2k.deg <= 2) rw2[5 + 2 * l2k.idx] = cl;
-                        else blk_ptr(D, l2k.b0)[l2k.idx].y = cl;
-                    }
-                    pp = l2k.link;
-                    if (--g2 < 0) { D.err = SAM_SEQ_WALK_LIMIT; return; }
-                }
+                redirect_walk(D, lk.link, t, q, cl, (int)plen + 2, ahead, na, nb2);
+                if (D.err) return;
             }
             if (D.lane == 0) reinterpret_cast<uint32_t*>(rq)[1] = cl;        // link[q] = cl
             __syncwarp();
@@ -469,7 +488,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             pa = make_uint4(plen + 1, qa.y, qa.z, qa.w); pb = nb;
         }
     }
-    if (D.lane == 0) D.text[ntok] = (int32_t)t;
+    if (D.lane == 0) { D.text[ntok] = (int32_t)t; D.pstate[ntok] = c; }
     last = c; ntok = k;
 }
 
@@ -505,12 +524,160 @@ __device__ __forceinline__ int dyn_fresh_run(Dyn& D, uint32_t tk, int j, int cnt
         }
         D.root[D.pr_slot] = make_uint2(tk, c | (plen == 0 ? SAM_FLAG : 0u));
         D.text[plen] = (int32_t)tk;
+        D.pstate[plen] = c;
     }
     const unsigned run = ((r >= 32 ? 0u : (1u << r)) - 1u) << j;
     if (bucket_peers & run) D.pr_state = 0;                   // those buckets changed
     __syncwarp();
     D.n_states = c0 + r; D.root_deg += r;
     last = c0 + r - 1; ntok += r;
+    return r;
+}
+
+// A run of tokens that repeat a passage of the sequence and all make Expand clone (Algorithm 3).
+// While the match (state s2, length l0, first end position e) is extended by the tokens that followed
+// its earliest occurrence, token k of the run reaches q_k, a state with first end position e + 1 + k,
+// through a transition that is not solid: a new state c_k, a clone cl_k of q_k with length l0 + k + 1,
+// the transition of the previous clone pointed to cl_k, link[q_k] = cl_k.  One Expand after the other
+// finds q_k only from q_{k-1}'s record.  Here the q_k are guessed — the states of the prefixes ending at
+// e + 1 + k (position -> state map) when the passage occurred once before, ids two apart when q_0 is a
+// clone left by an earlier repeat — their records are read in one round trip, one lane per token, and
+// checked (q_{k-1}'s transition on token k must lead to the guessed q_k); the lanes then write their
+// new states side by side.  Only the redirect walks above each clone (they start at the old link of
+// q_{k-1}) run one after the other.  Writing every link[q_k] before the walks gives what one Expand
+// after the other gives: a walk of token k follows states shorter than l0 + k, every q_k' with k' > k
+// is longer, and what a walk reads ahead (its first record) is checked not to be a q_k.
+// On entry (pa, pb) is the record of s2.  Returns the number of tokens taken (0: not such a run; pre
+// then offers the records read on the way to the ordinary Expand of token j).
+__device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cnt, uint32_t& last, uint32_t& ntok,
+                                              uint32_t& s2, uint32_t& l2, uint4& pa, uint4& pb, Pre& pre,
+                                              uint32_t (*stage)[12]) {
+    pre.valid = false;
+    if (pa.w == 0 || pa.w > 2 || cnt - j < 2) return 0;
+    const int lane = D.lane;
+    const uint32_t t0 = __shfl_sync(FULL, tk, j);
+    int idx0; uint32_t qt;
+    if (pb.x == t0) { idx0 = 0; qt = pb.y; }
+    else if (pa.w == 2 && pb.z == t0) { idx0 = 1; qt = pb.w; }
+    else return 0;
+    if (qt & SAM_FLAG) return 0;                               // solid: Expand does not clone
+    const uint32_t q0 = qt, e = pa.z, l0 = l2, u0 = pa.y;
+    const int rmax = min(cnt - j, (int)(ntok - e));            // text[e + k] must exist already
+    if (rmax < 2) return 0;
+    __syncwarp();
+
+    // round 1: the text after the earlier occurrence and the states created there; the records of q_0
+    // and of link[s2] (what the ordinary Expand of token j would read, should this not be a run)
+    const uint32_t tkr = __shfl_sync(FULL, tk, (j + lane) & 31);          // lane k: token k of the run
+    const uint32_t tnext = __shfl_sync(FULL, tk, (j + lane + 1) & 31);
+    int32_t tx = -1; uint32_t ps = SAM_NONE;
+    if (lane < rmax) { tx = D.text[e + lane]; ps = D.pstate[e + lane]; }
+    const uint4* rq0 = rec_ptr(D, q0);
+    const uint4* ru0 = rec_ptr(D, u0 ? u0 : q0);
+    uint4 qa = rq0[0], qb = rq0[1], ua = make_uint4(0, 0, 0, 0), ub = ua;
+    if (u0) { ua = ru0[0]; ub = ru0[1]; }
+    const unsigned same = __ballot_sync(FULL, lane < rmax && (uint32_t)tx == tkr);
+    // q_0 may be `last` itself (if token j does not continue the earliest occurrence), whose record is
+    // only completed by the Expand of token j: what was read of it is then not used
+    if (q0 != last) {
+        uint4* keep = reinterpret_cast<uint4*>(&stage[0][0]);
+        if (lane == 0) { keep[0] = qa; keep[1] = qb; keep[2] = ua; keep[3] = ub; }
+        __syncwarp();
+        pre.valid = true; pre.q = q0; pre.rec = keep;
+    }
+    int r = (~same) ? __ffs(~same) - 1 : 32;
+    if (r < 2) return 0;
+    // Where the q_k are expected: the states of the prefixes ending there if the passage occurred once
+    // before (q_0 is then the prefix state); otherwise q_0 is a clone from an earlier repeat of the
+    // passage, and clones made token after token have ids two apart.  Either guess is checked below.
+    if (__shfl_sync(FULL, ps, 0) != q0) ps = q0 + 2 * (uint32_t)lane;
+
+    // round 2: the records of q_1 .. q_{r-1} (states that exist and are complete: not `last`)
+    const bool exists = ps < D.n_states && ps != last;
+    {
+        const bool rd = lane > 0 && lane < r && exists;
+        const uint4* rqk = rec_ptr(D, rd ? ps : q0);
+        if (rd) { qa = rqk[0]; qb = rqk[1]; }
+    }
+    // q_k: inline transitions only, first end position e + 1 + k, reached by a transition that is not
+    // solid; and, but for the last of the run, its transition on the next token leads to q_{k+1}
+    int nidx = -1;
+    if (qa.w >= 1 && qa.w <= 2 && qb.x == tnext) nidx = 0;
+    else if (qa.w == 2 && qb.z == tnext) nidx = 1;
+    const uint32_t ntgt = (nidx == 0 ? qb.y : qb.w) & SAM_IDMASK;
+    const uint32_t psn = __shfl_down_sync(FULL, ps, 1);
+    const unsigned okm = __ballot_sync(FULL, lane < r && exists && qa.w <= 2 && qa.z == e + 1 + (uint32_t)lane &&
+                                                 qa.x > l0 + 1 + (uint32_t)lane);
+    const unsigned nxm = __ballot_sync(FULL, nidx >= 0 && ntgt == psn);
+    r = min(r, (~okm) ? __ffs(~okm) - 1 : 32);
+    r = min(r, ((~nxm) ? __ffs(~nxm) - 1 : 32) + 1);
+    if (r < 2) return 0;
+
+    // round 3: where each redirect walk starts, the old link of q_{k-1} (of s2 for k = 0)
+    uint32_t u = __shfl_up_sync(FULL, qa.y, 1);
+    if (lane == 0) u = u0;
+    {
+        const bool rd = lane > 0 && lane < r && u != 0;
+        const uint4* ruk = rec_ptr(D, rd ? u : q0);
+        if (rd) { ua = ruk[0]; ub = ruk[1]; }
+    }
+    {   // a walk's first record has been read now, before link[q_k] changes: it must not be one of the
+        // q_k (the q_k are told apart by their first end positions e + 1 + k)
+        const int kk = (int)ua.z - (int)e - 1;
+        const uint32_t cand = __shfl_sync(FULL, ps, kk & 31);
+        const unsigned inq = __ballot_sync(FULL, lane < r && u != 0 && kk >= 0 && kk < r && cand == u);
+        if (inq) r = min(r, __ffs(inq) - 1);
+        if (r < 2) return 0;
+    }
+
+    *reinterpret_cast<uint4*>(&stage[lane][0]) = ua;
+    *reinterpret_cast<uint4*>(&stage[lane][4]) = ub;
+    *reinterpret_cast<uint4*>(&stage[lane][8]) = make_uint4(tkr, ps, u, 0);
+
+    const uint32_t n0 = D.n_states;                            // c_k = n0 + 2k, cl_k = n0 + 2k + 1
+    ensure_rec(D, n0);
+    if (!D.err) ensure_rec(D, n0 + 2 * (uint32_t)r - 1);
+    if (D.err) return 0;
+
+    // the new states, side by side
+    const bool mine = lane < r;
+    const uint32_t ck = n0 + 2 * (uint32_t)lane, clk = ck + 1;
+    uint4* rprev = rec_ptr(D, mine ? (lane == 0 ? last : ck - 2) : 1u);      // the state whose transition t_k leaves
+    uint4* rcl = rec_ptr(D, mine ? clk : 1u);
+    uint32_t* rqw = reinterpret_cast<uint32_t*>(rec_ptr(D, mine ? ps : 1u));
+    uint32_t* rs2 = reinterpret_cast<uint32_t*>(rec_ptr(D, s2));
+    uint4 nb = make_uint4(qb.x, qb.y & SAM_IDMASK, qb.z, qb.w & SAM_IDMASK);  // copies are never solid ...
+    if (lane < r - 1) {                                                       // ... until redirected to the next clone
+        if (nidx == 0) nb.y = (clk + 2) | SAM_FLAG; else nb.w = (clk + 2) | SAM_FLAG;
+    }
+    if (mine) {
+        rprev[0] = make_uint4(ntok + lane, lane == 0 ? s2 : clk - 2, ntok + lane, 1);
+        rprev[1] = make_uint4(tkr, ck | SAM_FLAG, 0, 0);
+        rcl[0] = make_uint4(l0 + 1 + lane, qa.y, qa.z, qa.w);
+        rcl[1] = nb;
+        rqw[1] = clk;                                                         // link[q_k] = cl_k
+        D.text[ntok + lane] = (int32_t)tkr;
+        D.pstate[ntok + lane] = ck;
+        if (lane == 0) rs2[5 + 2 * idx0] = clk | SAM_FLAG;                    // s2's transition on t_0
+    }
+    __syncwarp();
+
+    // the redirect walks, one after the other; what each needs was left in shared memory by its lane
+    for (int k = 0; k < r && !D.err; k++) {
+        D.cur = j + k;
+        const uint4 xa = *reinterpret_cast<const uint4*>(&stage[k][0]);
+        const uint4 xb = *reinterpret_cast<const uint4*>(&stage[k][4]);
+        const uint4 xc = *reinterpret_cast<const uint4*>(&stage[k][8]);       // token, q_k, start of the walk
+        redirect_walk(D, xc.z, xc.x, xc.y, n0 + 2 * (uint32_t)k + 1, (int)(l0 + k) + 2, xc.z != 0, xa, xb);
+    }
+    if (D.err) return 0;
+
+    const int lr = r - 1;                                      // the last clone is the new match state
+    pa = make_uint4(l0 + (uint32_t)r, __shfl_sync(FULL, qa.y, lr), __shfl_sync(FULL, qa.z, lr), __shfl_sync(FULL, qa.w, lr));
+    pb = make_uint4(__shfl_sync(FULL, nb.x, lr), __shfl_sync(FULL, nb.y, lr), __shfl_sync(FULL, nb.z, lr), __shfl_sync(FULL, nb.w, lr));
+    D.n_states = n0 + 2 * (uint32_t)r;
+    last = n0 + 2 * (uint32_t)lr; s2 = last + 1; l2 = l0 + (uint32_t)r; ntok += (uint32_t)r;
+    pre.valid = false;
     return r;
 }
 
@@ -538,6 +705,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __shared__ int32_t sh_l[2], sh_s[2], sh_dl[2], sh_err[2];
+    __shared__ __align__(16) uint32_t sh_run[32][12];   // per-token staging of a repeat run (dynamic warp)
 
     // Everything the step needs to get going is read in one round trip: the slot's 64 control
     // words (state, slab table, copies of the two match states' records), its count, and the
@@ -697,6 +865,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         D.pool = A.W.pool;
         D.root = A.W.root_tab + (size_t)b * A.W.root_cap;
         D.text = A.W.text + (size_t)b * A.W.text_stride;
+        D.pstate = A.W.pstate + (size_t)b * A.W.text_stride;
         D.pool_hdr = A.W.pool_hdr; D.free_stack = A.W.free_stack; D.slab_owner = A.W.slab_owner;
         D.cb = cb;
         {   // slab table entry i is control word 16 + i
@@ -731,8 +900,15 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                     if (r > 0) { j += r; have = false; continue; }
                     if (D.err) break;
                 }
+                Pre pre;
+                pre.valid = false;
+                if (s2 != 0 && have) {
+                    const int r = dyn_repeat_run(D, tk, j, cnt, last, ntok, s2, l2, ra, rb, pre, sh_run);
+                    if (r > 0) { j += r; continue; }
+                    if (D.err) break;
+                }
                 D.cur = j;
-                dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2, have, ra, rb);
+                dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2, have, ra, rb, pre);
                 j++;
             }
         }
