@@ -10,8 +10,8 @@ struct sam_static {
     int device;
     void* dev_base;               // one allocation holding every section
     size_t dev_bytes;
-    size_t off_rec, off_root, off_hash, off_corpus, off_freq, off_topk;   // section offsets in dev_base
-    size_t len_rec, len_root, len_hash, len_corpus, len_freq, len_topk;   // section sizes in bytes
+    size_t off_rec, off_root, off_hash, off_corpus, off_freq, off_topk, off_pstate;   // section offsets in dev_base
+    size_t len_rec, len_root, len_hash, len_corpus, len_freq, len_topk, len_pstate;   // section sizes in bytes
     SamStaticView view;
     sam_static_info_t info;
 };

@@ -13,6 +13,10 @@
 //               hash(state, tok) & mask, overflow goes to the following buckets.  An empty entry
 //               has state == SAM_NONE; a bucket with an empty entry ends a probe sequence.
 //   corpus    : the int32 token text, padded so vector reads past the end stay in bounds.
+//   pstate    : uint32 per corpus token: id | F of the state Build-SAM created for it (the state of the
+//               whole prefix).  A match that is in such a state occurs exactly once in the corpus, so
+//               it continues exactly as the corpus does and its states can be read from this array
+//               instead of one record after the other.  Derived on the device after each upload.
 //   freq, topk: optional, for tree drafts — the occurrence count of every state, and for states
 //               with hashed transitions their k most frequent successors (a state with at most two
 //               transitions has them all in its record).
@@ -107,6 +111,7 @@ struct SamStaticView {
     const uint4* topk;        // SamTopkEnt table, four 16-byte words per entry
     uint32_t topk_mask;       // entries - 1
     int32_t tree_k;           // successors kept per hashed state (0: no tree data)
+    const uint32_t* pstate;   // [n_tokens]: id | F of the state of the prefix ending with corpus token i
 };
 
 // Device-side view of a batch workspace.

@@ -40,6 +40,9 @@ void layout_sections(sam_static* st) {
     st->off_corpus = off; off = sam_align_up(off + st->len_corpus, 256);
     st->off_freq = off;   off = sam_align_up(off + st->len_freq, 256);
     st->off_topk = off;   off = sam_align_up(off + st->len_topk, 256);
+    // derived on the device after every upload, never stored in a file: position -> prefix state
+    st->len_pstate = sam_align_up(((size_t)st->info.n_tokens + CORPUS_PAD_TOKENS) * 4, 8);
+    st->off_pstate = off; off = sam_align_up(off + st->len_pstate, 256);
     st->dev_bytes = off;
 }
 
@@ -58,6 +61,27 @@ void make_view(sam_static* st) {
     st->view.topk = (const uint4*)(base + st->off_topk);
     st->view.topk_mask = st->len_topk ? (uint32_t)(st->len_topk / sizeof(SamTopkEnt) - 1) : 0;
     st->view.tree_k = st->info.tree_topk;
+    st->view.pstate = (const uint32_t*)(base + st->off_pstate);
+}
+
+// pstate[i] = id | F of the state Build-SAM created for corpus token i, the state of the whole prefix
+// of length i + 1.  These are the states that are not clones: exactly those with len == min_endpos.
+__global__ void derive_pstate_kernel(const uint4* rec, int64_t n_states, uint32_t* pstate, int64_t n_tokens) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t s = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; s < n_states; s += stride) {
+        const uint4 a = rec[2 * s];
+        if (s > 0 && a.x == a.z && a.x >= 1 && (int64_t)a.x <= n_tokens)
+            pstate[a.x - 1] = (uint32_t)s | (a.w > 2 ? SAM_FLAG : 0u);
+    }
+}
+
+int derive_pstate(sam_static* st) {
+    derive_pstate_kernel<<<148 * 8, 256>>>(st->view.rec, st->info.n_states,
+                                           (uint32_t*)((char*)st->dev_base + st->off_pstate), st->info.n_tokens);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
+    return SAM_OK;
 }
 
 // collect the transitions of one state: inline ones, hashed ones, or the root row
@@ -165,6 +189,7 @@ extern "C" int sam_build_static(const int32_t* corpus_host, int64_t n_tokens, in
     if (e == cudaSuccess && !img.topk.empty()) e = cudaMemcpy(base + st->off_topk, img.topk.data(), st->len_topk, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { sam_set_cuda_error(e); cudaFree(st->dev_base); delete st; return SAM_ERR_CUDA; }
     make_view(st);
+    if (derive_pstate(st) != SAM_OK) { cudaFree(st->dev_base); delete st; return SAM_ERR_CUDA; }
     *out = st;
     return SAM_OK;
 }
@@ -281,6 +306,7 @@ extern "C" int sam_static_load(const char* path, int device, sam_static_t** out)
     if (rc == SAM_OK && sum != h.checksum) rc = SAM_ERR_FORMAT;
     if (rc != SAM_OK) { cudaFree(st->dev_base); delete st; return rc; }
     make_view(st);
+    if (derive_pstate(st) != SAM_OK) { cudaFree(st->dev_base); delete st; return SAM_ERR_CUDA; }
     *out = st;
     return SAM_OK;
 }

@@ -792,7 +792,35 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
             uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
             int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
             bool have = s != 0;
-            for (int base = 0; base < m && !err; base += 32) {
+            // A match whose state is the state of a whole corpus prefix (len == min_endpos: not a clone)
+            // occurs exactly once in the corpus, ending at e.  Its only transition is the next corpus
+            // token, and leads to the state of the prefix one longer.  So the tokens are compared with
+            // the corpus after e and the state is taken from the position -> state array, all in one
+            // round trip, in which the draft after e + m is requested as well in case every token agrees.
+            int j0 = 0;                      // tokens already taken
+            bool drafted = false;
+            if (have && m >= 1 && m <= 32 && ra.x == ra.z) {
+                const int64_t e = (int64_t)ra.z;
+                int32_t cx = -2; uint32_t px = 0;
+                if (lane < m && e + lane < A.S.n_tokens) { cx = __ldg(A.S.corpus + e + lane); px = __ldg(A.S.pstate + e + lane); }
+                const int64_t e2 = e + m;
+                const int64_t room = A.S.n_tokens - e2;
+                const int dl2 = (int)(room < L ? (room < 0 ? 0 : room) : L);
+                gather_draft<true>(A.S.corpus, e2, dl2, L, lane, d);
+                const unsigned agree = __ballot_sync(FULL, lane < m && cx == tok_first);
+                j0 = (~agree) ? __ffs(~agree) - 1 : 32;
+                if (j0 > 0) {
+                    const uint32_t ref = __shfl_sync(FULL, px, j0 - 1);
+                    s = ref & SAM_IDMASK; sf = ref >> 31; l += j0; have = false;
+                    if (j0 == m) {                                  // the whole step: the draft is in already
+                        ra = __ldg(A.S.rec + 2 * (size_t)s);        // its record, for the next step
+                        rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
+                        my_dl = cut_at_stop(d, dl2, lane, A.W.stop_token);
+                        drafted = true;
+                    }
+                }
+            }
+            for (int base = 0; base < m && !err && j0 < m; base += 32) {
                 const int i = base + lane;
                 uint32_t tk = 0, re = SAM_NONE;
                 if (i < m) { tk = (uint32_t)(base == 0 ? tok_first : toks[i]); re = __ldg(A.S.root_row + tk); }
@@ -818,7 +846,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                             sp_ent[r] = __ldg(A.S.hash + (size_t)(sam_hash2(u, tnext) & A.S.hash_mask) * SAM_HASH_BUCKET + e);
                     }
                 }
-                for (int j = 0; j < cnt && !err; j++) {
+                for (int j = j0; j < cnt && !err; j++) {
                     bool pre = false;
                     uint4 pa = ra, pb = rb, pent = make_uint4(SAM_NONE, 0, 0, 0);
                     if (j >= 1 && j <= 8 && s != 0) {
@@ -843,7 +871,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
                 }
             }
             my_l = l; my_s = (int32_t)s;
-            if (l > 0 && !err) {
+            if (l > 0 && !err && !drafted) {
                 if (m > 0) {                                    // the state moved: read its record, keep a copy
                     ra = __ldg(A.S.rec + 2 * (size_t)s);
                     rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
