@@ -469,7 +469,7 @@ def main_ours(args):
         "e2e": {"value": units_all / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": B * spec.accept_max * 4 + B * 4, "d2h_bytes_per_step": B * (L + 7) * 4,
                 "ms_per_step": e2e_ms / K, "api": "sam_step_host"},
-        "gpu_launches": K,
+        "gpu_launches": K * batch.launches_per_step(),
         "graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms / K, "value": units / (graph_ms * 1e-3),
                                                        "note": "the K sam_step launches captured in one CUDA graph"},
         "clocks": clocks,

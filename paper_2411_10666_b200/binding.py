@@ -75,6 +75,7 @@ SIGNATURES = {
     "sam_batch_dump": (c_int, [c_void_p, c_int32, _i32p, _i32p, _i32p, c_void_p, c_void_p, c_void_p, c_void_p,
                                c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p]),
     "sam_batch_pool_info": (c_int, [c_void_p, POINTER(c_int64), POINTER(c_int64), c_void_p]),
+    "sam_batch_launches_per_step": (c_int, [c_void_p]),
     "sam_batch_destroy": (None, [c_void_p]),
     "sam_accept_greedy": (c_int, [c_int32, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32,
                                   c_void_p, c_void_p, c_void_p]),
@@ -456,6 +457,11 @@ class Batch:
 
     def pool_info(self):
         return sam_batch_pool_info(self.handle)
+
+    def launches_per_step(self) -> int:
+        n = lib().sam_batch_launches_per_step(self.handle)
+        _check(n if n < 0 else SAM_OK, "sam_batch_launches_per_step")
+        return n
 
     def close(self):
         if getattr(self, "handle", None):

@@ -13,7 +13,7 @@ constexpr size_t SAM_ZERO_COPY_MAX_BYTES = 256u << 10;   // larger host steps go
 constexpr int SAM_POLL_LIMIT_US = 2000;                  // how long a host step polls its completion flag
 
 struct WsLayout {
-    size_t off_hdr, off_ctrl, off_free, off_owner, off_reset, off_text, off_pstate, off_root, off_stage, off_pool, total;
+    size_t off_hdr, off_ctrl, off_free, off_owner, off_reset, off_order, off_text, off_pstate, off_root, off_stage, off_pool, total;
     int32_t text_stride, root_cap, slab_shift, pool_slabs, max_host_stride;
     size_t stage_words;
 };
@@ -52,6 +52,7 @@ int plan(const sam_batch_opts_t* o, WsLayout* w) {
     w->off_free = off;  off = sam_align_up(off + (size_t)slabs * 4, 256);
     w->off_owner = off; off = sam_align_up(off + (size_t)slabs * 4, 256);
     w->off_reset = off; off = sam_align_up(off + (size_t)o->batch * 4 * 2, 256);   // flags + slot list
+    w->off_order = off; off = sam_align_up(off + (size_t)o->batch * 4 * 2, 256);
     w->off_text = off;  off = sam_align_up(off + (size_t)o->batch * w->text_stride * 4, 256);
     w->off_pstate = off; off = sam_align_up(off + (size_t)o->batch * w->text_stride * 4, 256);
     w->off_root = off;  off = sam_align_up(off + (size_t)o->batch * w->root_cap * 8, 256);
@@ -173,6 +174,7 @@ int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBa
         view->free_stack = (int32_t*)(b + w.off_free);
         view->slab_owner = (int32_t*)(b + w.off_owner);
         view->reset_flag = (int32_t*)(b + w.off_reset);
+        view->order = (int32_t*)(b + w.off_order);
         view->text = (int32_t*)(b + w.off_text);
         view->pstate = (uint32_t*)(b + w.off_pstate);
         view->root_tab = (uint2*)(b + w.off_root);
@@ -240,6 +242,7 @@ extern "C" int sam_batch_create(const sam_static_t* st, const sam_batch_opts_t* 
     V.free_stack = (int32_t*)(base + w.off_free);
     V.slab_owner = (int32_t*)(base + w.off_owner);
     V.reset_flag = (int32_t*)(base + w.off_reset);
+    V.order = (int32_t*)(base + w.off_order);
     V.text = (int32_t*)(base + w.off_text);
     V.pstate = (uint32_t*)(base + w.off_pstate);
     V.root_tab = (uint2*)(base + w.off_root);
@@ -416,6 +419,11 @@ extern "C" int sam_step_host(sam_batch_t* b, const int32_t* new_tokens_host, int
     if (state_host) memcpy(state_host, ho + B * L + 4 * B, 2 * B * 4);
     memcpy(status_host, ho + B * L + 6 * B, B * 4);
     return SAM_OK;
+}
+
+extern "C" int sam_batch_launches_per_step(const sam_batch_t* b) {
+    if (!b) return SAM_ERR_ARG;
+    return sam_step_launch_count(b);
 }
 
 extern "C" int sam_batch_pool_info(sam_batch_t* b, int64_t* total_slabs, int64_t* free_slabs, void* stream) {

@@ -27,6 +27,7 @@ struct sam_batch {
     int32_t* host_stage;          // pinned, device-mapped host staging area
     int32_t* host_stage_dev;      // the same memory as the device addresses it
     int32_t host_seq;             // sequence number of the last host-array step (completion flag value)
+    mutable int32_t order_phase;  // which of the two slot-order buffers the next large-batch step uses
 };
 
 void sam_set_cuda_error(cudaError_t e);
@@ -66,6 +67,9 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
                          int32_t* done_flag_dev, int32_t done_seq,
                          const int32_t* v_draft, const int32_t* v_draft_len, const int32_t* v_max_new,
                          int32_t* v_counts_out, int32_t* v_accepted_out);
+
+// 1, or 2 when the batch is large enough for the slot-ordering kernel (step.cu)
+int sam_step_launch_count(const sam_batch* b);
 
 // helpers implemented in batch.cu
 int sam_plan_view(const sam_batch_opts_t* opts, int32_t vocab, void* base, SamBatchView* view,

@@ -121,6 +121,7 @@ struct SamBatchView {
     int32_t* free_stack;      // [pool_slabs]
     int32_t* slab_owner;      // [pool_slabs], -1 = free
     int32_t* reset_flag;      // [B]
+    int32_t* order;           // [2][B]: slots sorted by their step's token count (large batches), two buffers in turn
     int32_t* text;            // [B][text_stride]
     uint32_t* pstate;         // [B][text_stride]: id of the state created by each text position
     uint2* root_tab;          // [B][root_cap]

@@ -19,7 +19,14 @@
 //     entries of all tokens of the step, and the dynamic root-table lookups of all tokens of a chunk,
 //     one lane per token;
 //   - runs of tokens that are new to the sequence while nothing is matched are extended by the lanes
-//     in parallel (each such Expand is three independent writes).
+//     in parallel (each such Expand is three independent writes);
+//   - runs of tokens that repeat a passage of the sequence and make every Expand clone are extended by
+//     the lanes in parallel as well: the states the clones are made from are guessed (position -> state
+//     map, or ids two apart), read in one round trip and checked (dyn_repeat_run);
+//   - a static match that occurs only once in the corpus is advanced by comparing the step's tokens with
+//     the corpus, its state read from the corpus' position -> state array;
+//   - when the batch is larger than the GPU holds at once, the slots with the most tokens are started
+//     first (order_slots_kernel).
 #include "common.h"
 
 #include <cstring>
@@ -44,6 +51,8 @@ struct StepArgs {
     // derived here: the confirmed prefix of its previous draft plus the target's next token
     const int32_t* v_draft; const int32_t* v_draft_len; const int32_t* v_max_new;
     int32_t* v_counts_out; int32_t* v_accepted_out;
+    // optional: block i works on slot order[i] (slots with many tokens first; see order_slots_kernel)
+    const int32_t* order;
 };
 
 // ------------------------------------------------------------------ draft read
@@ -702,7 +711,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     // after this one is allowed to get scheduled right away (it waits in the same way).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
-    const int b = blockIdx.x;
+    const int b = A.order ? A.order[blockIdx.x] : (int)blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __shared__ int32_t sh_l[2], sh_s[2], sh_dl[2], sh_err[2];
     __shared__ __align__(16) uint32_t sh_run[32][12];   // per-token staging of a repeat run (dynamic warp)
@@ -1001,7 +1010,41 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     }
 }
 
+// A batch larger than the GPU holds at once runs in waves, and a step is as long as its last block: a
+// slot with many tokens that starts in the last wave ends late.  This kernel sorts the slots by their
+// token count, largest first (a counting sort in shared memory), so that block i of the step kernel takes
+// slot order[i] and the long slots start in the first wave.  It reads only the step's counts, so it runs
+// while the step before is still going; it ends with griddepcontrol.wait, so that its own completion —
+// all the next step kernel waits for — implies that of the step before.
+constexpr int SAM_ORDER_KEYS = 64;
+__global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts, int32_t B, int32_t* order) {
+    asm volatile("griddepcontrol.launch_dependents;");
+    __shared__ int hist[SAM_ORDER_KEYS];
+    for (int k = threadIdx.x; k < SAM_ORDER_KEYS; k += blockDim.x) hist[k] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < B; i += blockDim.x) {
+        const int m = counts[i];
+        atomicAdd(&hist[m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m)], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {                                  // hist[k] <- first position of key k, keys descending
+        int at = 0;
+        for (int k = SAM_ORDER_KEYS - 1; k >= 0; k--) { const int n = hist[k]; hist[k] = at; at += n; }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < B; i += blockDim.x) {
+        const int m = counts[i];
+        const int pos = atomicAdd(&hist[m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m)], 1);
+        order[pos] = i;
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+constexpr int SAM_ORDER_MIN_BATCH = 1536;                    // more slots than a B200 holds blocks of this kernel (148 x 10)
+
 }  // namespace
+
+int sam_step_launch_count(const sam_batch* b) { return b->view.batch >= SAM_ORDER_MIN_BATCH ? 2 : 1; }
 
 int sam_launch_step(const sam_batch* b, const int32_t* new_tokens, int32_t stride, const int32_t* counts,
                     int32_t L, int32_t* draft_tokens, int32_t* draft_len, int32_t* match_len,
@@ -1035,12 +1078,23 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
     A.new_tokens = new_tokens; A.stride = stride; A.counts = counts; A.L = L;
     A.draft_tokens = draft_tokens; A.draft_len = draft_len; A.match_len = match_len;
     A.source = source; A.state = state; A.status = status;
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3((unsigned)b->view.batch); cfg.blockDim = dim3(64); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    A.order = nullptr;
+    if (!v_draft && b->view.batch >= SAM_ORDER_MIN_BATCH) {
+        int32_t* order = b->view.order + (size_t)(b->order_phase & 1) * b->view.batch;
+        b->order_phase ^= 1;
+        cudaLaunchConfig_t oc;
+        memset(&oc, 0, sizeof(oc));
+        oc.gridDim = dim3(1); oc.blockDim = dim3(1024); oc.stream = stream; oc.attrs = attr; oc.numAttrs = 1;
+        cudaError_t oe = cudaLaunchKernelEx(&oc, order_slots_kernel, counts, (int32_t)b->view.batch, order);
+        if (oe != cudaSuccess) { sam_set_cuda_error(oe); return SAM_ERR_CUDA; }
+        A.order = order;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)b->view.batch); cfg.blockDim = dim3(64); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
     cfg.attrs = attr; cfg.numAttrs = 1;
     cudaError_t e = v_draft ? cudaLaunchKernelEx(&cfg, sam_step_kernel<true>, A)
                             : cudaLaunchKernelEx(&cfg, sam_step_kernel<false>, A);

@@ -142,6 +142,96 @@ def test_adversarial_sequences(P):
         assert_dynamic_automata_equal(batch, ob, [0], n)
 
 
+def test_repeated_passages_dynamic_runs(P):
+    """Passages repeated once, twice and three times, with contexts of different lengths before them,
+    self-overlapping repeats, periodic stretches and repeats of the very beginning of the text: the
+    cases in which the step kernel extends several cloning tokens side by side.  Every output and the
+    whole automaton equal the oracle's."""
+    rng = random.Random(11)
+    n = 1400
+    for vocab, kmax in [(3, 40), (6, 32), (50, 17), (2000, 40), (2000, 3)]:
+        x = [rng.randrange(vocab) for _ in range(60)]
+        while len(x) < n:
+            kind = rng.random()
+            if kind < 0.45:                                   # repeat an earlier span (again and again)
+                s = rng.randrange(len(x)); ln = rng.randint(2, 70)
+                x.extend(x[s:s + ln])
+            elif kind < 0.55:                                 # overlap: the span runs into itself
+                back = rng.randint(1, 12); ln = rng.randint(5, 60)
+                for _ in range(ln):
+                    x.append(x[-back])
+            elif kind < 0.62:                                 # the beginning of the text once more
+                x.extend(x[:rng.randint(2, 50)])
+            else:
+                x.extend(rng.randrange(vocab) for _ in range(rng.randint(1, 6)))
+        x = x[:n]
+        nt, ct = _steps_from_text(x, rng, kmax)
+        empty = np.zeros((1, 0), np.int32)
+        for L in (1, 32):
+            ref, ob, _ = oracle_run(None, vocab, empty, nt, ct, L, n)
+            got, batch = gpu_run(P, None, vocab, empty, nt, ct, L, n)
+            assert_same(got, ref, "vocab %d kmax %d L %d" % (vocab, kmax, L))
+            assert_dynamic_automata_equal(batch, ob, [0], n)
+            assert (got["status"] == 0).all()
+
+
+def test_static_matches_in_prefix_states(P):
+    """Sequences that copy long stretches of the corpus (the match soon occurs only once, so the static
+    side advances it by comparing with the corpus), including stretches that run to the corpus' end,
+    that break off after any number of tokens, and a corpus with internal repeats."""
+    rng = random.Random(12)
+    for vocab, N in [(4, 300), (40, 5000), (3000, 20000)]:
+        corpus = []
+        while len(corpus) < N:
+            if corpus and rng.random() < 0.2:
+                s = rng.randrange(len(corpus)); corpus.extend(corpus[s:s + rng.randint(3, 40)])
+            else:
+                corpus.append(rng.randrange(vocab))
+        corpus = np.array(corpus[:N], dtype=np.int32)
+        n = 900
+        texts = []
+        for b in range(3):
+            x = []
+            while len(x) < n:
+                r = rng.random()
+                if r < 0.5:
+                    s = rng.randrange(N); x.extend(corpus[s:s + rng.randint(1, 90)].tolist())
+                elif r < 0.6:
+                    x.extend(corpus[N - rng.randint(1, 50):].tolist())          # up to the corpus' end
+                else:
+                    x.extend(rng.randrange(vocab) for _ in range(rng.randint(1, 4)))
+            texts.append(x[:n])
+        kmax = 32
+        rows, cnts, k = [], [], 0
+        while k < n:
+            m = min(rng.randint(0, kmax), n - k)
+            rows.append([t[k:k + m] + [-1] * (kmax - m) for t in texts]); cnts.append([m] * 3); k += m
+        nt = np.array(rows, dtype=np.int32).reshape(len(rows), 3, kmax)
+        ct = np.array(cnts, dtype=np.int32).reshape(len(rows), 3)
+        empty = np.zeros((3, 0), np.int32)
+        st = P.StaticSam.build(corpus, vocab)
+        for L, stop in ((8, -1), (40, 1)):
+            ref, ob, _ = oracle_run(corpus, vocab, empty, nt, ct, L, n, stop_token=stop)
+            got, batch = gpu_run(P, st, vocab, empty, nt, ct, L, n, stop_token=stop)
+            assert_same(got, ref, "vocab %d N %d L %d" % (vocab, N, L))
+            assert (got["source"] == 1).any()
+
+
+def test_large_batch_is_ordered_by_token_count(P):
+    """A batch above the size at which the step first sorts its slots by token count (two kernels per
+    step): the results are the same as the oracle's, slot for slot."""
+    spec = W.scaled(W.SPECS["c5"], 150_000, 1700, 48, 80)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, ob, _ = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=4)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    assert batch.launches_per_step() == 2
+    assert_same(got, ref, "ordered batch")
+    assert (got["status"] == 0).all()
+    assert_dynamic_automata_equal(batch, ob, [0, 777, spec.batch - 1], msl)
+
+
 CASES = {
     # name: (spec key, corpus_len, batch, prompt_len, gen_len) — same recipes, smaller sizes
     "tiny_full": ("tiny", None, None, None, None),
