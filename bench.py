@@ -46,7 +46,7 @@ ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of sam_step_kernel from the committed ncu
 # capture (profiles/ncu_full_sam_step_kernel_c2.md); None for workloads without a capture of the
 # kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 178005}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 179797}
 
 
 def parse_args():
