@@ -575,7 +575,7 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
     if (rmax < 2) return 0;
     __syncwarp();
 
-    // round 1: the text after the earlier occurrence and the states created there; the records of q_0
+    // first round trip: the text after the earlier occurrence and the states created there; the records of q_0
     // and of link[s2] (what the ordinary Expand of token j would read, should this not be a run)
     const uint32_t tkr = __shfl_sync(FULL, tk, (j + lane) & 31);          // lane k: token k of the run
     const uint32_t tnext = __shfl_sync(FULL, tk, (j + lane + 1) & 31);
@@ -601,7 +601,7 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
     // passage, and clones made token after token have ids two apart.  Either guess is checked below.
     if (__shfl_sync(FULL, ps, 0) != q0) ps = q0 + 2 * (uint32_t)lane;
 
-    // round 2: the records of q_1 .. q_{r-1} (states that exist and are complete: not `last`)
+    // second round trip: the records of q_1 .. q_{r-1} (states that exist and are complete: not `last`)
     const bool exists = ps < D.n_states && ps != last;
     {
         const bool rd = lane > 0 && lane < r && exists;
@@ -622,7 +622,7 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
     r = min(r, ((~nxm) ? __ffs(~nxm) - 1 : 32) + 1);
     if (r < 2) return 0;
 
-    // round 3: where each redirect walk starts, the old link of q_{k-1} (of s2 for k = 0)
+    // third round trip: where each redirect walk starts, the old link of q_{k-1} (of s2 for k = 0)
     uint32_t u = __shfl_up_sync(FULL, qa.y, 1);
     if (lane == 0) u = u0;
     {

@@ -68,7 +68,7 @@ def try_run(S, toks, deg_limit=2):
     # the guess: prefix states after e, or ids two apart from q0
     ps = [S.pstate[e + k] if S.pstate[e] == q0 else q0 + 2 * k for k in range(r)]
     rec = []
-    for k in range(r):                                       # round 2: records, read before any write
+    for k in range(r):                                       # second read: the records, before any write
         if ps[k] >= len(S.len) or ps[k] == S.last:
             r = k
             break
@@ -95,7 +95,7 @@ def try_run(S, toks, deg_limit=2):
                 break
     if r < 2:
         return 0
-    first = [dict(S.next[x]) if x > 0 else None for x in u[:r]]   # round 3, still before any write
+    first = [dict(S.next[x]) if x > 0 else None for x in u[:r]]   # third read, still before any write
     n0, last = len(S.len), S.last
     for k in range(r):                                       # new states, side by side
         S.new(ntok + k + 1, -1, ntok + k + 1, {})
