@@ -189,8 +189,8 @@ int sam_step(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
 /* Replay n_steps consecutive steps from device arrays without returning to the caller in
  * between: new_tokens_dev [n_steps, B, stride], counts_dev [n_steps, B].  If out_per_step is
  * non-zero every output array has a leading n_steps dimension and keeps each step's results,
- * otherwise the arrays are those of sam_step and hold the last step's.  One kernel launch per
- * step, same kernel as sam_step. */
+ * otherwise the arrays are those of sam_step and hold the last step's.  The launches of each
+ * step are those sam_step makes (sam_batch_launches_per_step). */
 int sam_run_steps(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
                   const int32_t* counts_dev, int32_t n_steps, int32_t L, int32_t out_per_step,
                   int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,
