@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--workload", default="c2", choices=sorted(W.SPECS))
     ap.add_argument("--min-seconds", type=float, default=2.5, help="keep repeating the timed region this long")
     ap.add_argument("--max-repeats", type=int, default=300)
+    ap.add_argument("--batch", type=int, default=0,
+                    help="run the workload's recipe with this many sequences per GPU instead of its own batch (a scaling probe, not a headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probes", action="store_true")
     ap.add_argument("--tree-draft", action="store_true",
@@ -283,6 +285,8 @@ def main_ours(args):
     P.lib()
 
     base = W.SPECS[args.workload]
+    if args.batch > 0:
+        base = W.scaled(base, batch=args.batch)
     spec, corpus, seqs, counts, new_tokens = shard_workload(base, rank, world)
     B, L = seqs.shape[0], spec.draft_len
     msl = spec.prompt_len + spec.gen_len
@@ -427,7 +431,7 @@ def main_ours(args):
     except Exception:
         peak = 6650.0
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(base.name), "peak_source": peak_src + " stream copy",
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(base.name) if args.batch <= 0 else None, "peak_source": peak_src + " stream copy",
                 "kernel": "sam_step_kernel", "launch_us": launch_us,
                 "algorithmic_bytes_per_sequence_step": algo_b,
                 "sequence_steps_per_launch": units / K}
@@ -452,7 +456,7 @@ def main_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32", "data": "synthetic",
-        "config": {"workload": base.name, "batch_per_gpu": B, "global_batch": B * world,
+        "config": {"workload": base.name + ("" if args.batch <= 0 else " (recipe run with %d sequences)" % args.batch), "batch_per_gpu": B, "global_batch": B * world,
                    "prompt_len": spec.prompt_len, "gen_len": spec.gen_len, "draft_len": L,
                    "corpus_tokens": spec.corpus_len, "vocab": spec.vocab,
                    "static_states": int(info.n_states), "static_bytes": int(info.device_bytes),
