@@ -692,8 +692,12 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
 
 // Called by one thread of a block after the block's outputs are written (and made known to that
 // thread by a block barrier where another warp wrote some of them).
+// A block orders its output stores (to mapped host memory) before its count with a device-scope fence;
+// the block that counts last has thereby observed all the others, and its one system-scope fence — fences
+// are cumulative — orders every block's stores before the flag the host polls.  (A system-scope fence in
+// every block is what the host waited for: 3.5 us more at 64 blocks, 7 us more at 256.)
 __device__ __forceinline__ void signal_done(const StepArgs& A) {
-    __threadfence_system();
+    __threadfence();
     const int prev = atomicAdd(A.done_count, 1);
     if (prev == (int)gridDim.x - 1) {
         *A.done_count = 0;
