@@ -198,9 +198,13 @@ int sam_run_steps(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
 
 /* sam_step with HOST arrays: copies new_tokens and counts to the device, runs the step, copies
  * every output back and waits for the stream — the end-to-end call a serving loop that keeps its
- * tokens on the host would make.  stride <= max_host_stride.  Pinned host buffers make the
- * copies asynchronous with respect to other streams; pageable ones work too.  state_host may be
- * NULL.  Synchronous.  Errors: as sam_step, plus CUDA. */
+ * tokens on the host would make.  stride <= max_host_stride.  Any host memory works.  How the
+ * bytes travel depends on the step's size: small steps go through a page-locked staging area that
+ * the kernel reads and writes itself; from 64 KiB of arrays on, arrays that are ALL page-locked and
+ * device-addressable (cudaHostAlloc, cudaHostRegister, a pinned torch tensor) are read and written
+ * in place by the kernel, and any others are copied through the staging area.  state_host may be
+ * NULL.  Synchronous: the results are in the arrays when the call returns.  Errors: as sam_step,
+ * plus CUDA. */
 int sam_step_host(sam_batch_t* b, const int32_t* new_tokens_host, int32_t stride,
                   const int32_t* counts_host, int32_t L,
                   int32_t* draft_tokens_host, int32_t* draft_len_host, int32_t* match_len_host,

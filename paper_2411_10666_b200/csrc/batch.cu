@@ -9,7 +9,8 @@
 
 namespace {
 
-constexpr size_t SAM_ZERO_COPY_MAX_BYTES = 256u << 10;   // larger host steps go through two DMA copies
+constexpr size_t SAM_ZERO_COPY_MAX_BYTES = 4u << 20;     // larger host steps go through two DMA copies
+constexpr size_t SAM_DIRECT_MIN_BYTES = 64u << 10;       // from this size on, page-locked caller arrays are used in place
 constexpr int SAM_POLL_LIMIT_US = 2000;                  // how long a host step polls its completion flag
 
 struct WsLayout {
@@ -379,6 +380,36 @@ extern "C" int sam_step_host(sam_batch_t* b, const int32_t* new_tokens_host, int
     int32_t* hst = b->host_stage;
     const size_t in_words = B * stride + B;
     const size_t out_words = B * L + 7 * B;
+    if ((in_words + out_words) * 4 >= SAM_DIRECT_MIN_BYTES) {
+        // Large steps: copying the arrays through the staging area on the host costs more than the step.
+        // If every array the caller passed is page-locked memory the device can address (cudaHostAlloc /
+        // cudaHostRegister: what a pinned torch tensor is), the kernel reads and writes them in place.
+        const void* hp[8] = {new_tokens_host, counts_host, draft_tokens_host, draft_len_host, match_len_host,
+                             source_host, status_host, state_host};
+        void* dp[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+        bool direct = true;
+        for (int i = 0; i < 8 && direct; i++) {
+            if (!hp[i]) continue;                              // state_host may be null
+            if (cudaHostGetDevicePointer(&dp[i], const_cast<void*>(hp[i]), 0) != cudaSuccess) { cudaGetLastError(); direct = false; }
+        }
+        if (direct) {
+            volatile int32_t* flag = b->host_stage + b->stage_words;
+            const int32_t seq = ++b->host_seq == 0 ? ++b->host_seq : b->host_seq;
+            rc = sam_launch_step_signal(b, (const int32_t*)dp[0], stride, (const int32_t*)dp[1], L, (int32_t*)dp[2], (int32_t*)dp[3],
+                                        (int32_t*)dp[4], (int32_t*)dp[5], (int32_t*)dp[7], (int32_t*)dp[6], s,
+                                        b->host_stage_dev + b->stage_words, seq);
+            if (rc) return rc;
+            const auto t0 = std::chrono::steady_clock::now();
+            bool seen = false;
+            for (uint32_t spin = 0;; spin++) {
+                if (*flag == seq) { seen = true; break; }
+                if ((spin & 1023u) == 1023u &&
+                    std::chrono::steady_clock::now() - t0 > std::chrono::microseconds(SAM_POLL_LIMIT_US)) break;
+            }
+            if (!seen) SAM_CUDA(cudaStreamSynchronize(s));
+            return SAM_OK;
+        }
+    }
     memcpy(hst, new_tokens_host, B * stride * 4);
     memcpy(hst + B * stride, counts_host, B * 4);
     int32_t* ho = hst + in_words;

@@ -146,6 +146,33 @@ def test_host_step_equals_device_step(P):
         P.binding.sam_step_host(b.handle, big, big.shape[1], np.zeros(B, np.int32), L, *[out[k] for k in KEYS])
 
 
+@pytest.mark.parametrize("B", [600, 1700])
+def test_host_step_large_with_pinned_and_pageable_arrays(P, B):
+    """Large host steps: page-locked caller arrays are read and written in place, pageable ones go
+    through the staging area (and, at this size, two DMA copies or the mapped staging area); at 1700
+    slots the slot-ordering kernel reads the counts from host memory too.  All equal the oracle."""
+    import torch
+    spec = W.scaled(W.SPECS["c5"], corpus_len=60_000, batch=B, prompt_len=24, gen_len=40)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, _, _ = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=4)
+    steps = [(w.prompts, np.full(B, spec.prompt_len, dtype=np.int32))] + \
+            [(w.new_tokens[s], w.counts[s]) for s in range(w.n_steps)]
+    for pinned in (True, False):
+        b = P.Batch(st, B, msl, max_draft_len=L, max_host_stride=spec.prompt_len)
+        mk = (lambda *s: torch.empty(s, dtype=torch.int32).pin_memory()) if pinned else (lambda *s: torch.empty(s, dtype=torch.int32))
+        out = dict(draft_tokens=mk(B, L), draft_len=mk(B), match_len=mk(B, 2), source=mk(B), state=mk(B, 2), status=mk(B))
+        for i, (toks, cnt) in enumerate(steps):
+            t = torch.from_numpy(np.ascontiguousarray(toks)); c = torch.from_numpy(np.ascontiguousarray(cnt))
+            if pinned:
+                t, c = t.pin_memory(), c.pin_memory()
+            P.binding.sam_step_host(b.handle, t, t.shape[1], c, L, *[out[k] for k in KEYS])
+            for k in KEYS:
+                assert np.array_equal(out[k].numpy(), ref[k][i]), (pinned, i, k)
+        b.close()
+
+
 def test_image_save_load_roundtrip(P, tmp_path):
     spec = W.scaled(W.SPECS["c2"], corpus_len=120_000, batch=4, prompt_len=100, gen_len=200)
     w = W.make(spec)
