@@ -266,6 +266,23 @@ def sam_step_host(h, new_tokens, stride, counts, L, draft_tokens, draft_len, mat
            "sam_step_host")
 
 
+def sam_step_host_prepared(h, stride, L, draft_tokens, draft_len, match_len, source, state, status, stream=None):
+    """The same call as sam_step_host for a loop that makes it every step: whatever does not change
+    from step to step (the output arrays, stride, L, the stream) is converted once, and the returned
+    function takes the step's new_tokens and counts (arrays, or plain addresses)."""
+    fn = lib().sam_step_host
+    fixed = [c_void_p(_host_ptr(x, n)) for x, n in ((draft_tokens, "draft_tokens"), (draft_len, "draft_len"),
+                                                     (match_len, "match_len"), (source, "source"), (state, "state"),
+                                                     (status, "status"))]
+    sp, hh = c_void_p(_stream_ptr(stream)), c_void_p(h) if isinstance(h, int) else h
+
+    def call(new_tokens, counts):
+        rc = fn(hh, _host_ptr(new_tokens, "new_tokens"), stride, _host_ptr(counts, "counts"), L, *fixed, sp)
+        if rc != SAM_OK:
+            raise SamError(rc, "sam_step_host")
+    return call
+
+
 def sam_batch_dump(h, slot: int, max_states: int, max_edges: int, stream=None):
     nt, ns, ne = c_int32(), c_int32(), c_int32()
     st = [np.zeros(max(max_states, 1), dtype=np.int32) for _ in range(4)]

@@ -135,10 +135,16 @@ def test_host_step_equals_device_step(P):
     out = dict(draft_tokens=mk(B, L), draft_len=mk(B), match_len=mk(B, 2), source=mk(B), state=mk(B, 2), status=mk(B))
     steps = [(w.prompts, np.full(B, spec.prompt_len, dtype=np.int32))] + \
             [(w.new_tokens[s], w.counts[s]) for s in range(w.n_steps)]
+    prepared = {}                                       # the bound form of the call, one per stride
     for i, (toks, cnt) in enumerate(steps):
         toks = np.ascontiguousarray(toks)
-        P.binding.sam_step_host(b.handle, toks, toks.shape[1], np.ascontiguousarray(cnt), L,
-                                *[out[k] for k in KEYS])
+        if i % 2 == 0:
+            P.binding.sam_step_host(b.handle, toks, toks.shape[1], np.ascontiguousarray(cnt), L,
+                                    *[out[k] for k in KEYS])
+        else:
+            if toks.shape[1] not in prepared:
+                prepared[toks.shape[1]] = P.binding.sam_step_host_prepared(b.handle, toks.shape[1], L, *[out[k] for k in KEYS])
+            prepared[toks.shape[1]](toks, np.ascontiguousarray(cnt))
         for k in KEYS:
             assert np.array_equal(out[k].numpy(), ref[k][i]), (i, k)
     with pytest.raises(P.SamError):
