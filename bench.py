@@ -43,10 +43,11 @@ UNIT = "sequence-steps/s"
 # and the input and output rows.
 ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.1}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of sam_step_kernel from the committed ncu
-# capture (profiles/ncu_full_sam_step_kernel_c2.md); None for workloads without a capture of the
-# kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 179797}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of sam_step_kernel (median of 60 launches) from the
+# committed one-pass ncu capture that leaves the caches as the loop leaves them
+# (profiles/ncu_dram_traffic_warm_sam_step_kernel_c2.md; the cold-cache capture of --set full shows 179797);
+# None for workloads without a capture of the kernel as it stands.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 98944}
 
 
 def parse_args():
