@@ -713,6 +713,16 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     // Programmatic dependent launch: this grid may be scheduled while the previous kernel of the stream
     // is still finishing.  Nothing is read before that kernel has completed and flushed; the kernel
     // after this one is allowed to get scheduled right away (it waits in the same way).
+    if (!A.order) {
+        // While the previous kernel of the stream finishes: touch (prefetch, no data is used) the lines this
+        // block reads first, so that their address translations and L2 lines are at hand after the wait.
+        const int pb_ = blockIdx.x, pl_ = threadIdx.x & 31;
+        const char* p0 = reinterpret_cast<const char*>(A.W.ctrl + (size_t)pb_ * SAM_CTRL_WORDS);
+        const char* p1 = reinterpret_cast<const char*>(A.new_tokens + (size_t)pb_ * A.stride);
+        const char* p2 = reinterpret_cast<const char*>(VERIFY ? A.v_draft_len + pb_ : A.counts + pb_);
+        const char* pp_ = pl_ == 0 ? p0 : pl_ == 1 ? p0 + 128 : pl_ == 2 ? p1 : p2;
+        if (pl_ < 4) asm volatile("prefetch.global.L2 [%0];" ::"l"(pp_));
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const int b = A.order ? A.order[blockIdx.x] : (int)blockIdx.x;
