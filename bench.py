@@ -45,9 +45,9 @@ ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of sam_step_kernel (median of 60 launches) from the
 # committed one-pass ncu capture that leaves the caches as the loop leaves them
-# (profiles/ncu_dram_traffic_warm_sam_step_kernel_c2.md; the cold-cache capture of --set full shows 179797);
+# (profiles/ncu_dram_traffic_warm_sam_step_kernel_c2.md; the cold-cache capture of --set full shows 179115);
 # None for workloads without a capture of the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 98944}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 94336}
 
 
 def parse_args():
