@@ -180,7 +180,14 @@ int sam_batch_reset(sam_batch_t* b, const int32_t* slots_host, int32_t n, void* 
  * Host-visible argument errors (null, L out of range, stride < 1) return ARG synchronously and
  * launch nothing; data-dependent problems are reported per slot in status_dev and freeze the
  * slot until it is reset.  A slot is validated (count, capacity, token range) before any of its
- * state changes. */
+ * state changes.
+ *
+ * Stream order is all the call needs: new_tokens_dev and counts_dev may be written by the kernel
+ * that precedes this call on `stream` (sam_accept_greedy, sam_step_verified's counts_out_dev, the
+ * caller's own kernel).  The step reads them only after everything earlier on the stream has
+ * completed.  For batches that take two launches (sam_batch_launches_per_step), the first launch
+ * looks at counts_dev early, possibly before they are final, but only to decide in which order
+ * the slots are started; no result depends on what it saw. */
 int sam_step(sam_batch_t* b, const int32_t* new_tokens_dev, int32_t stride,
              const int32_t* counts_dev, int32_t L,
              int32_t* draft_tokens_dev, int32_t* draft_len_dev, int32_t* match_len_dev,

@@ -14,9 +14,12 @@
 //               has state == SAM_NONE; a bucket with an empty entry ends a probe sequence.
 //   corpus    : the int32 token text, padded so vector reads past the end stay in bounds.
 //   pstate    : uint32 per corpus token: id | F of the state Build-SAM created for it (the state of the
-//               whole prefix).  A match that is in such a state occurs exactly once in the corpus, so
-//               it continues exactly as the corpus does and its states can be read from this array
-//               instead of one record after the other.  Derived on the device after each upload.
+//               whole prefix ending there; exactly the states with len == min_endpos).  The transition
+//               of such a state on the next corpus token is solid and therefore never redirected: it
+//               leads to the next entry of this array.  A match that sits in a prefix state and goes on
+//               as the corpus does can take its states from this array instead of one record after the
+//               other; a token that differs from the corpus takes the ordinary Transfer (the state may
+//               well have other transitions and other occurrences).  Derived on the device after each upload.
 //   freq, topk: optional, for tree drafts — the occurrence count of every state, and for states
 //               with hashed transitions their k most frequent successors (a state with at most two
 //               transitions has them all in its record).
@@ -121,7 +124,7 @@ struct SamBatchView {
     int32_t* free_stack;      // [pool_slabs]
     int32_t* slab_owner;      // [pool_slabs], -1 = free
     int32_t* reset_flag;      // [B]
-    int32_t* order;           // [2][B]: slots sorted by their step's token count (large batches), two buffers in turn
+    int32_t* order;           // [3][B]: slots sorted by their step's token count (large batches), two buffers in turn; then the sort keys
     int32_t* text;            // [B][text_stride]
     uint32_t* pstate;         // [B][text_stride]: id of the state created by each text position
     uint2* root_tab;          // [B][root_cap]

@@ -74,7 +74,7 @@ extern "C" int sam_retrieve_noalloc(const sam_static_t* st, int32_t vocab, int32
     rc = scratch_for_device(device, &base);
     if (rc) return rc;
 
-    sam_batch tmp;                                            // lives for this call only; nothing is allocated
+    sam_batch tmp{};                                          // lives for this call only; nothing is allocated
     tmp.device = device; tmp.st = st; tmp.opts = o; tmp.workspace_bytes = need;
     tmp.max_host_stride = 0; tmp.stage_words = 0; tmp.host_stage = nullptr; tmp.host_stage_dev = nullptr; tmp.host_seq = 0;
     rc = sam_plan_view(&o, o.vocab, base, &tmp.view, nullptr, nullptr);

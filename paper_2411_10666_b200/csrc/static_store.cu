@@ -76,9 +76,12 @@ __global__ void derive_pstate_kernel(const uint4* rec, int64_t n_states, uint32_
 }
 
 int derive_pstate(sam_static* st) {
-    derive_pstate_kernel<<<148 * 8, 256>>>(st->view.rec, st->info.n_states,
+    int sms = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, st->device);
+    if (e != cudaSuccess || sms < 1) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
+    derive_pstate_kernel<<<sms * 8, 256>>>(st->view.rec, st->info.n_states,
                                            (uint32_t*)((char*)st->dev_base + st->off_pstate), st->info.n_tokens);
-    cudaError_t e = cudaGetLastError();
+    e = cudaGetLastError();
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
     return SAM_OK;

@@ -23,8 +23,9 @@
 //   - runs of tokens that repeat a passage of the sequence and make every Expand clone are extended by
 //     the lanes in parallel as well: the states the clones are made from are guessed (position -> state
 //     map, or ids two apart), read in one round trip and checked (dyn_repeat_run);
-//   - a static match that occurs only once in the corpus is advanced by comparing the step's tokens with
-//     the corpus, its state read from the corpus' position -> state array;
+//   - a static match that sits in the state of a whole corpus prefix is advanced by comparing the step's
+//     tokens with the corpus, its state read from the corpus' position -> state array (a prefix state's
+//     transition on the next corpus token always leads to the next prefix state);
 //   - when the batch is larger than the GPU holds at once, the slots with the most tokens are started
 //     first (order_slots_kernel).
 #include "common.h"
@@ -815,11 +816,15 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
             uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
             int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
             bool have = s != 0;
-            // A match whose state is the state of a whole corpus prefix (len == min_endpos: not a clone)
-            // occurs exactly once in the corpus, ending at e.  Its only transition is the next corpus
-            // token, and leads to the state of the prefix one longer.  So the tokens are compared with
-            // the corpus after e and the state is taken from the position -> state array, all in one
-            // round trip, in which the draft after e + m is requested as well in case every token agrees.
+            // The match state is the state Build-SAM created for a whole corpus prefix (len == min_endpos:
+            // not a clone), the prefix ending at e.  Its transition on the next corpus token was created
+            // solid (len + 1) and a solid transition is never redirected, so it still leads to the state of
+            // the prefix one longer, with match length l + 1.  The state may occur more than once and have
+            // other transitions too ("ab" in "ababc"): nothing is assumed about those.  The step's tokens
+            // are compared with the corpus after e; as long as they agree the state is taken from the
+            // position -> state array, and the first token that differs goes through the ordinary Transfer
+            // below.  All in one round trip, in which the draft after e + m is requested as well in case
+            // every token agrees.
             int j0 = 0;                      // tokens already taken
             bool drafted = false;
             if (have && m >= 1 && m <= 32 && ra.x == ra.z) {
@@ -1030,15 +1035,23 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
 // slot order[i] and the long slots start in the first wave.  It reads only the step's counts, so it runs
 // while the step before is still going; it ends with griddepcontrol.wait, so that its own completion —
 // all the next step kernel waits for — implies that of the step before.
+// The counts may still be changing while this kernel reads them (when the kernel before it on the stream
+// is the one that writes them), so each count is read exactly once: the key taken from it is kept in
+// `keys` and used for both passes.  order[] is therefore a permutation of the slots whatever was read;
+// a count read too early only costs the intended launch order, never a result (the step kernel reads the
+// counts itself, after its own dependency wait).
 constexpr int SAM_ORDER_KEYS = 64;
-__global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts, int32_t B, int32_t* order) {
+__global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts, int32_t B, int32_t* order,
+                                                           int32_t* keys) {
     asm volatile("griddepcontrol.launch_dependents;");
     __shared__ int hist[SAM_ORDER_KEYS];
     for (int k = threadIdx.x; k < SAM_ORDER_KEYS; k += blockDim.x) hist[k] = 0;
     __syncthreads();
     for (int i = threadIdx.x; i < B; i += blockDim.x) {
-        const int m = counts[i];
-        atomicAdd(&hist[m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m)], 1);
+        const int m = *reinterpret_cast<const volatile int32_t*>(counts + i);
+        const int key = m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m);
+        keys[i] = key;                                       // read back by this same thread below
+        atomicAdd(&hist[key], 1);
     }
     __syncthreads();
     if (threadIdx.x == 0) {                                  // hist[k] <- first position of key k, keys descending
@@ -1047,9 +1060,8 @@ __global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts
     }
     __syncthreads();
     for (int i = threadIdx.x; i < B; i += blockDim.x) {
-        const int m = counts[i];
-        const int pos = atomicAdd(&hist[m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m)], 1);
-        order[pos] = i;
+        const int pos = atomicAdd(&hist[keys[i]], 1);
+        if (pos < B) order[pos] = i;                         // always true: the keys are those counted above
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
@@ -1102,7 +1114,8 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
         cudaLaunchConfig_t oc;
         memset(&oc, 0, sizeof(oc));
         oc.gridDim = dim3(1); oc.blockDim = dim3(1024); oc.stream = stream; oc.attrs = attr; oc.numAttrs = 1;
-        cudaError_t oe = cudaLaunchKernelEx(&oc, order_slots_kernel, counts, (int32_t)b->view.batch, order);
+        cudaError_t oe = cudaLaunchKernelEx(&oc, order_slots_kernel, counts, (int32_t)b->view.batch, order,
+                                            b->view.order + 2 * (size_t)b->view.batch);
         if (oe != cudaSuccess) { sam_set_cuda_error(oe); return SAM_ERR_CUDA; }
         A.order = order;
     }

@@ -125,3 +125,97 @@ def test_fused_verify_and_step_matches_the_two_call_loop(P):
     assert np.array_equal(pos.cpu().numpy(), pos_ref)
     with pytest.raises(P.SamError):                                  # the previous draft may not be the output buffer
         P.binding.sam_step_verified(batch.handle, target, new.draft_tokens, new.draft_len, cap, L, *new.tensors())
+
+
+def _large_loop_case():
+    spec = W.scaled(W.SPECS["c5"], 150_000, 1600, 40, 60)
+    w = W.make(spec)
+    return spec, w
+
+
+def test_two_call_loop_above_the_slot_ordering_threshold(P):
+    """The closed loop with a batch large enough for the slot-ordering kernel (two launches per step):
+    the counts each step reads were written by the kernel just before it on the stream
+    (sam_accept_greedy), which is the case the ordering kernel must tolerate.  Step for step equal to
+    the oracle's loop."""
+    import torch
+    spec, w = _large_loop_case()
+    B, pl, L = spec.batch, spec.prompt_len, spec.draft_len
+    total, stride = pl + spec.gen_len, L + 1
+    S = oracle.Sam(w.corpus)
+    ob = oracle.Batch(S, w.corpus, B, spec.vocab, total)
+    log, pos_ref = accept.decode_loop(ob, w.seqs, pl, L, stride)
+
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    batch = P.Batch(st, B, total, max_draft_len=L)
+    assert batch.launches_per_step() == 2
+    dev = batch.device
+    seqs = _t(w.seqs, dev).long()
+    out = batch.step(_t(w.prompts, dev), torch.full((B,), pl, dtype=torch.int32, device=dev), L)
+    pos = torch.full((B,), pl, dtype=torch.int64, device=dev)
+    nt = torch.empty((B, stride), dtype=torch.int32, device=dev)
+    cnt = torch.empty(B, dtype=torch.int32, device=dev); acc = torch.empty_like(cnt)
+    ar = torch.arange(L + 1, device=dev)[None, :]
+    kept = []
+    for step in range(len(log)):                              # no host read inside the loop
+        target = torch.gather(seqs, 1, torch.clamp(pos[:, None] + ar, max=total - 1)).int().contiguous()
+        cap = (total - pos).int().contiguous()
+        P.binding.sam_accept_greedy(out.draft_tokens, out.draft_len, target, cap, nt, cnt, acc)
+        kept.append({k: getattr(out, k).clone() for k in ("draft_tokens", "draft_len", "match_len", "source", "state", "status")})
+        kept[-1]["counts"] = cnt.clone(); kept[-1]["accepted"] = acc.clone()
+        out = batch.step(nt, cnt, L, out)
+        pos += cnt.long()
+    torch.cuda.synchronize()
+    for step, ref in enumerate(log):
+        for k, v in kept[step].items():
+            assert np.array_equal(v.cpu().numpy(), ref[k]), (step, k)
+    assert np.array_equal(pos.cpu().numpy(), pos_ref) and (pos_ref == total).all()
+
+
+def test_counts_written_by_the_fused_step_feed_a_plain_step(P):
+    """sam_step_verified writes counts_out; the very next call on the stream is a sam_step that takes
+    that array as its counts (feeding as many tokens of the continuation again).  With 1600 slots the
+    plain step sorts its slots by those counts first.  Every output equals the oracle fed the same way."""
+    import torch
+    spec, w = _large_loop_case()
+    B, pl, L = spec.batch, spec.prompt_len, spec.draft_len
+    total = pl + spec.gen_len
+    S = oracle.Sam(w.corpus)
+    ob = oracle.Batch(S, w.corpus, B, spec.vocab, total)
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    batch = P.Batch(st, B, total, max_draft_len=L)
+    dev = batch.device
+    seqs = _t(w.seqs, dev).long()
+    outs = [P.StepOutputs(B, L, dev) for _ in range(3)]
+    batch.step(_t(w.prompts, dev), torch.full((B,), pl, dtype=torch.int32, device=dev), L, outs[0])
+    r_out = ob.step(w.prompts, np.full(B, pl, dtype=np.int32), L)
+    pos = torch.full((B,), pl, dtype=torch.int64, device=dev)
+    r_pos = np.full(B, pl, dtype=np.int64)
+    cnt = torch.empty(B, dtype=torch.int32, device=dev); acc = torch.empty_like(cnt)
+    ar = torch.arange(L + 1, device=dev)[None, :]
+    prev = outs[0]
+    for it in range(12):
+        mid, new = outs[(2 * it + 1) % 3], outs[(2 * it + 2) % 3]
+        # device: verify + update, then a plain step whose counts are the array the first kernel wrote
+        target = torch.gather(seqs, 1, torch.clamp(pos[:, None] + ar, max=total - 1)).int().contiguous()
+        cap = ((total - pos) // 2).int().contiguous()
+        P.binding.sam_step_verified(batch.handle, target, prev.draft_tokens, prev.draft_len, cap, L,
+                                    *mid.tensors(), counts_out=cnt, accepted_out=acc)
+        again = torch.gather(seqs, 1, torch.clamp(pos[:, None] + cnt.long()[:, None] + ar, max=total - 1)).int().contiguous()
+        batch.step(again, cnt, L, new)
+        pos += 2 * cnt.long()
+        # oracle, the same two updates
+        idx = np.minimum(r_pos[:, None] + np.arange(L + 1)[None, :], total - 1)
+        r_nt, r_cnt, r_acc = accept.accept_greedy(r_out.draft_tokens, r_out.draft_len,
+                                                  np.take_along_axis(w.seqs, idx, axis=1), (total - r_pos) // 2, L + 1)
+        r_mid = ob.step(r_nt, r_cnt, L)
+        idx2 = np.minimum(r_pos[:, None] + r_cnt[:, None] + np.arange(L + 1)[None, :], total - 1)
+        r_new = ob.step(np.ascontiguousarray(np.take_along_axis(w.seqs, idx2, axis=1)), r_cnt, L)
+        r_pos += 2 * r_cnt
+        assert np.array_equal(cnt.cpu().numpy(), r_cnt) and np.array_equal(acc.cpu().numpy(), r_acc), it
+        gm, gn = mid.cpu(), new.cpu()
+        for k in ("draft_tokens", "draft_len", "match_len", "source", "state", "status"):
+            assert np.array_equal(gm[k], getattr(r_mid, k)), (it, "verified", k)
+            assert np.array_equal(gn[k], getattr(r_new, k)), (it, "plain", k)
+        prev, r_out = new, r_new
+    assert np.array_equal(pos.cpu().numpy(), r_pos) and (r_pos > pl).all()

@@ -176,10 +176,14 @@ def test_repeated_passages_dynamic_runs(P):
 
 
 def test_static_matches_in_prefix_states(P):
-    """Sequences that copy long stretches of the corpus (the match soon occurs only once, so the static
-    side advances it by comparing with the corpus), including stretches that run to the corpus' end,
-    that break off after any number of tokens, and a corpus with internal repeats."""
+    """Sequences that copy long stretches of the corpus (the match soon sits in the state of a whole
+    corpus prefix, so the static side advances it by comparing with the corpus), including stretches
+    that run to the corpus' end, that break off after any number of tokens, and corpora with internal
+    repeats.  The periodic corpora ("abab...", "ababc", period 3 with a tail) have prefix states that
+    occur several times and have two transitions — the state of "ab" in "ababc" goes on with a and
+    with c — so tokens that leave the corpus' own continuation from such a state are covered."""
     rng = random.Random(12)
+    made = []
     for vocab, N in [(4, 300), (40, 5000), (3000, 20000)]:
         corpus = []
         while len(corpus) < N:
@@ -187,8 +191,15 @@ def test_static_matches_in_prefix_states(P):
                 s = rng.randrange(len(corpus)); corpus.extend(corpus[s:s + rng.randint(3, 40)])
             else:
                 corpus.append(rng.randrange(vocab))
-        corpus = np.array(corpus[:N], dtype=np.int32)
-        n = 900
+        made.append((vocab, corpus[:N]))
+    made.append((3, [0, 1, 0, 1, 2]))                                     # ababc
+    made.append((3, [0, 1] * 40))                                         # (ab)^40
+    made.append((3, [0, 1] * 30 + [2] + [0, 1] * 20 + [2, 2, 0]))         # two periodic stretches
+    made.append((4, [0, 1, 2] * 25 + [3] + [0, 1, 2, 0, 1, 3]))           # period 3 with tails
+    for vocab, corpus in made:
+        N = len(corpus)
+        corpus = np.array(corpus, dtype=np.int32)
+        n = 900 if N > 200 else 400
         texts = []
         for b in range(3):
             x = []
@@ -197,7 +208,9 @@ def test_static_matches_in_prefix_states(P):
                 if r < 0.5:
                     s = rng.randrange(N); x.extend(corpus[s:s + rng.randint(1, 90)].tolist())
                 elif r < 0.6:
-                    x.extend(corpus[N - rng.randint(1, 50):].tolist())          # up to the corpus' end
+                    x.extend(corpus[N - rng.randint(1, min(50, N)):].tolist())  # up to the corpus' end
+                elif r < 0.7:
+                    x.extend(corpus[:rng.randint(1, min(60, N))].tolist())      # from the corpus' start: prefix states
                 else:
                     x.extend(rng.randrange(vocab) for _ in range(rng.randint(1, 4)))
             texts.append(x[:n])

@@ -310,3 +310,34 @@ def test_stop_token_cuts_the_draft_at_a_document_separator():
             assert out.source[0] == exp["source"]
             assert out.draft_tokens[0, :dl].tolist() == d and (out.draft_tokens[0, dl:] == -1).all()
             assert EOS not in out.draft_tokens[0, :dl].tolist()
+
+
+@pytest.mark.parametrize("threads", [1, 3])
+def test_run_of_many_steps_equals_the_definition_and_the_single_steps(threads):
+    """Batch.run (all steps of a schedule in one call: what the timed CPU baseline executes) leaves,
+    for every sequence, exactly what exhaustive search gives for its whole text, and the same
+    outputs, automata and operation counts as feeding the steps one by one."""
+    rng = random.Random(77 + threads)
+    for _ in range(25):
+        vocab, B, K, L = rng.randint(2, 4), rng.randint(1, 4), rng.randint(1, 5), rng.randint(1, 6)
+        N, n_steps = rng.randint(0, 50), rng.randint(1, 14)
+        l_bias, min_match = rng.randint(0, 2), rng.randint(0, 2)
+        corpus = _random_text(rng, N, vocab)
+        counts = np.array([[rng.randint(0, K) for _ in range(B)] for _ in range(n_steps)], dtype=np.int32)
+        toks = np.array([[[rng.randrange(vocab) for _ in range(K)] for _ in range(B)] for _ in range(n_steps)], dtype=np.int32)
+        total = int(counts.sum(axis=0).max()) + 1
+        S = oracle.Sam(corpus) if N else None
+        whole = oracle.Batch(S, corpus if N else None, B, vocab, total, l_bias, min_match)
+        out = whole.run(toks, counts, L, threads)
+        single = oracle.Batch(S, corpus if N else None, B, vocab, total, l_bias, min_match)
+        for s in range(n_steps):
+            ref = single.step(toks[s], counts[s], L)
+        for k in ("draft_tokens", "draft_len", "match_len", "source", "state", "status"):
+            assert np.array_equal(getattr(out, k), getattr(ref, k)), k
+        assert whole.counters() == single.counters()
+        for b in range(B):
+            x = [int(t) for s in range(n_steps) for t in toks[s, b, :counts[s, b]]]
+            exp = bf.retrieve(corpus if N else None, x, len(x), L, l_bias, min_match)
+            assert out.match_len[b].tolist() == [exp["l1"], exp["l2"]] and out.source[b] == exp["source"]
+            assert out.draft_tokens[b, :out.draft_len[b]].tolist() == exp["draft"]
+            assert whole.seq_len(b) == len(x) and whole.dynamic(b).n_states == single.dynamic(b).n_states
