@@ -1,15 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the batched suffix-automaton draft-retrieval step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c5]
 
 A "step" is one `sam_step` over the whole batch: every slot feeds its accepted tokens of that
 decoding step through the static automaton (Transfer) and its own dynamic automaton
 (Transfer + Expand), the source is chosen and the draft is read.  The prompt prefill and W
 warm-up steps run untimed; then exactly K consecutive decoding steps of the schedule are timed
-with CUDA events (one kernel launch per step).  The K-step region is repeated from an identical
-state (reset, prefill, warm-up, L2 flush) until a few seconds have passed so that clock samples
-exist; the reported value is the median repeat.  One JSON line is printed by rank 0.
+with CUDA events.  The K-step region is repeated from an identical state (reset, prefill, warm-up,
+L2 flush) until a few seconds have passed so that clock samples exist; the reported value is the
+median repeat.  One JSON line is printed by rank 0.
+
+The headline workload is the largest of the five recipes (c5: 4096 sequences over a 200 M-token
+corpus).  At one GPU the line also carries `all_workloads`: the same measurement, shorter, for the
+other four recipes.  The CPU oracle is timed beside every workload on the same decoding steps; its
+automata are built in child processes while the GPU part runs (the builds are single-threaded and
+take minutes at 100-200 M tokens), and each child's timed run starts only when the GPU part is over.
 
 Under torchrun each rank owns a contiguous shard of a batch that is N times larger (weak scaling,
 the static automaton replicated, no collective on the data path); the time is the max over ranks.
@@ -17,6 +23,7 @@ the static automaton replicated, no collective on the data path); the time is th
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -35,44 +42,88 @@ import workloads as W  # noqa: E402
 
 METRIC = "sam_sequence_steps_per_sec"
 UNIT = "sequence-steps/s"
+HEADLINE = "c5"
+ORDER = ["tiny", "c2", "c3", "c4", "c5"]
 
-# Algorithmic bytes per sequence-step of the generation phase: what the method itself must read
-# and write, from the CPU oracle's operation counters (python -m oracle.count_ops <workload>):
-# 32 B per Transfer move, per walk-insert (+8 B edge), per clone (x2), per redirect (+4 B);
-# 32 B new state + 8 B links + 4 B text per token; per step two 32-B records, the drafted tokens
-# and the input and output rows.
-ALGO_BYTES = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.1}
+# Algorithmic bytes per sequence-step averaged over a recipe's whole generation phase (from the CPU
+# oracle's operation counters, `python -m oracle.count_ops <workload>`).  Used only when the oracle leg
+# is switched off; otherwise the bytes come from the oracle's counters over exactly the timed steps.
+ALGO_BYTES_WHOLE_PHASE = {"tiny": 750.3, "c2": 857.7, "c3": 935.1, "c4": 1374.8, "c5": 1024.1}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of sam_step_kernel (median of 60 launches) from the
-# committed one-pass ncu capture that leaves the caches as the loop leaves them
-# (profiles/ncu_dram_traffic_warm_sam_step_kernel_c2.md; the cold-cache capture of --set full shows 179115);
-# None for workloads without a capture of the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"c2": 94336}
+# DRAM traffic of one step launch (dram__bytes_read.sum + dram__bytes_write.sum, one-pass ncu capture that
+# leaves the caches as the loop leaves them), per capture: bytes per launch, sequence-steps per launch of
+# the captured case, and the digest of the kernel sources the capture was taken on.  A capture whose digest
+# is not that of the sources as they stand is not reported.
+NCU_TRAFFIC = {
+    # workload: (bytes per launch, slots per launch in the capture, source digest, note)
+}
+KERNEL_SOURCES = ("paper_2411_10666_b200/csrc/step.cu", "paper_2411_10666_b200/csrc/layout.h")
 
 
-def parse_args():
+def kernel_digest() -> str:
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=512)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(W.SPECS))
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(W.SPECS))
     ap.add_argument("--min-seconds", type=float, default=2.5, help="keep repeating the timed region this long")
     ap.add_argument("--max-repeats", type=int, default=300)
     ap.add_argument("--batch", type=int, default=0,
                     help="run the workload's recipe with this many sequences per GPU instead of its own batch (a scaling probe, not a headline)")
+    ap.add_argument("--corpus-tokens", type=int, default=0,
+                    help="run the workload's recipe over a corpus of this many tokens (a reduced case for profiler captures, not a headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probes", action="store_true")
+    ap.add_argument("--no-all-workloads", action="store_true", help="measure the named workload only")
+    ap.add_argument("--cpu-wait-seconds", type=float, default=900.0,
+                    help="how long to wait for an oracle automaton that is still being built")
+    ap.add_argument("--cache-dir", default=os.environ.get("SAMDRAFT_CACHE_DIR", ""),
+                    help="keep built static automata here between runs (sam_static_save / sam_static_load; the c5 image is "
+                         "18 GB); default: the SAMDRAFT_CACHE_DIR environment variable, else no caching")
     ap.add_argument("--tree-draft", action="store_true",
                     help="also time sam_tree_draft (builds the static automaton with top-k successor data)")
     ap.add_argument("--closed-loop", action="store_true",
                     help="also run draft -> verify -> accept -> update on the device with the true continuation as target")
-    return ap.parse_args()
+    return ap.parse_args(argv)
 
 
 def dist_env():
     return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
             int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def variant(name: str, batch: int = 0, corpus_tokens: int = 0) -> W.Spec:
+    spec = W.SPECS[name]
+    return W.scaled(spec, batch=batch or None, corpus_len=corpus_tokens or None)
+
+
+def config_dict(base: W.Spec, label: str, world: int) -> dict:
+    """What names the workload; the same for the GPU arm and the reference arm."""
+    return {"workload": label, "batch_per_gpu": base.batch, "global_batch": base.batch * world,
+            "prompt_len": base.prompt_len, "gen_len": base.gen_len, "draft_len": base.draft_len,
+            "accept_max": base.accept_max, "corpus_tokens": base.corpus_len, "vocab": base.vocab,
+            "parallelism": "batch-sharded x%d, static automaton replicated" % world,
+            "l2": "GPU arm: L2 flushed (288 MB write) before each timed region and the static store is larger than "
+                  "the 126 MB L2 except for the smallest recipes; per-sequence automata stay cache-warm between "
+                  "consecutive steps.  CPU arm: caches as the preceding steps leave them"}
+
+
+def workload_label(name: str, batch: int, corpus_tokens: int) -> str:
+    extra = []
+    if batch > 0:
+        extra.append("%d sequences" % batch)
+    if corpus_tokens > 0:
+        extra.append("%d corpus tokens" % corpus_tokens)
+    return name + (" (recipe run with %s)" % ", ".join(extra) if extra else "")
 
 
 class ClockSampler:
@@ -125,10 +176,11 @@ class ClockSampler:
         return out
 
 
-def shard_workload(spec: W.Spec, rank: int, world: int):
+def shard_workload(spec: W.Spec, rank: int, world: int, corpus=None):
     """Weak scaling: the global batch is `world` times the recipe's batch; this rank's shard."""
     big = W.scaled(spec, batch=spec.batch * world)
-    corpus = W.make_corpus(big)
+    if corpus is None:
+        corpus = W.make_corpus(big)
     seqs, counts, new_tokens = W.make_sequences(big, corpus, rank, world)
     return big, corpus, seqs, counts, new_tokens
 
@@ -147,24 +199,183 @@ def reduce_max_sum(local_ms: float, local_units: int, world: int):
     return float(t.item()), int(u.item())
 
 
-def run_oracle_timed(spec, corpus, seqs, counts, new_tokens, steps_lo, steps_hi, threads, static=None):
-    """Time the CPU oracle on decoding steps [steps_lo, steps_hi) after an untimed build, prefill
-    and the steps before steps_lo.  Returns (seconds, sequence-steps, draft tokens, automaton)."""
+# ---------------------------------------------------------------------------------------------
+# the CPU oracle, timed in a child process
+# ---------------------------------------------------------------------------------------------
+
+def algorithmic_bytes(c: dict, L: int) -> dict:
+    """Bytes the method itself must touch for the steps whose operation counts are `c`: a state is a
+    32-byte record; 32 B per Transfer move; per accepted token a new state (32 B), its two link fields
+    (8 B) and the text append (4 B); per walk-insert 32 B read + 8 B written; per clone 32 B read + 32 B
+    written; per redirect 32 B read + 4 B written; per step the two matched states' records, the drafted
+    tokens, the output row (4 L + 28 B) and the input row (4 m + 4 B)."""
+    steps, toks = max(c["seq_steps"], 1), c["tokens"]
+    static_b = 32 * (c["static_link_moves"] + c["static_next_moves"])
+    dyn_b = toks * 44 + c["walk_inserts"] * 40 + c["clones"] * 64 + c["redirects"] * 36
+    step_b = c["seq_steps"] * (64 + 4 * L + 28 + 4) + 4 * toks + 4 * c["draft_tokens"]
+    return {"static": static_b / steps, "dynamic": dyn_b / steps, "step_io": step_b / steps,
+            "total": (static_b + dyn_b + step_b) / steps}
+
+
+def dependent_accesses(c: dict) -> dict:
+    """Accesses per sequence-step that Algorithms 1 and 3 make one after the other (each needs the
+    result of the one before): on the static chain every Transfer move, then the matched state's record
+    and the draft; on the dynamic chain every link or next move of Transfer / Expand's walk, every clone
+    (the record of q) and redirect, then record and draft."""
+    steps = max(c["seq_steps"], 1)
+    st = (c["static_link_moves"] + c["static_next_moves"]) / steps + 2
+    dy = (c["dynamic_link_moves"] + c["dynamic_next_moves"] + c["clones"] + c["redirects"]) / steps + 2
+    return {"static_chain": st, "dynamic_chain": dy}
+
+
+def oracle_leg(base: W.Spec, Wm: int, K: int, threads: int, single_thread_budget_s: float = 8.0, wait_for_go=None, ready=None):
+    """Build the oracle's automata for `base`, run prefill and warm-up steps untimed, then time the K
+    decoding steps [Wm, Wm + K) on all `threads` cores (OpenMP over sequences, static automaton shared),
+    and a bounded share of them on one thread."""
     import oracle
-    S = static if static is not None else oracle.Sam(corpus)
-    B, L = seqs.shape[0], spec.draft_len
-    ob = oracle.Batch(S, corpus, B, spec.vocab, spec.prompt_len + spec.gen_len)
-    ob.step(np.ascontiguousarray(seqs[:, :spec.prompt_len]), np.full(B, spec.prompt_len, dtype=np.int32), L, threads)
-    if steps_lo > 0:
-        ob.run(new_tokens[:steps_lo], counts[:steps_lo], L, threads)
-    c0 = ob.counters()
+    few = max(1, min(4, threads // 4)) if wait_for_go is not None else threads   # untimed phases keep out of the GPU part's way
     t0 = time.perf_counter()
-    ob.run(new_tokens[steps_lo:steps_hi], counts[steps_lo:steps_hi], L, threads)
-    dt = time.perf_counter() - t0
+    corpus = W.make_corpus(base)
+    seqs, counts, new_tokens = W.make_sequences(base, corpus)
+    t1 = time.perf_counter()
+    S = oracle.Sam(corpus)
+    build_s = time.perf_counter() - t1
+    B, L = seqs.shape[0], base.draft_len
+    K = min(K, counts.shape[0] - Wm)
+    prompts = np.ascontiguousarray(seqs[:, :base.prompt_len])
+    pcount = np.full(B, base.prompt_len, dtype=np.int32)
+
+    def fresh():
+        ob = oracle.Batch(S, corpus, B, base.vocab, base.prompt_len + base.gen_len)
+        ob.step(prompts, pcount, L, few)
+        if Wm > 0:
+            ob.run(new_tokens[:Wm], counts[:Wm], L, few)
+        return ob
+
+    ob = fresh()
+    if ready is not None:
+        ready({"build_s": build_s, "inputs_s": t1 - t0})
+    if wait_for_go is not None:
+        wait_for_go()
+    few = threads                                        # the GPU part is over: use every core from here on
+    c0 = ob.counters()
+    t2 = time.perf_counter()
+    ob.run(new_tokens[Wm:Wm + K], counts[Wm:Wm + K], L, threads)
+    dt = time.perf_counter() - t2
     c1 = ob.counters()
     ob.close()
-    return dt, c1["seq_steps"] - c0["seq_steps"], c1["draft_tokens"] - c0["draft_tokens"], S
+    d = {k: c1[k] - c0[k] for k in c1}
+    units = d["seq_steps"]
+    res = {"value": units / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt, "steps": K,
+           "sequence_steps": units, "draft_tokens_per_sec": d["draft_tokens"] / dt,
+           "oracle_build_seconds": build_s, "counters": d,
+           "sample": "the same %d decoding steps x %d sequences (%d sequence-steps) as the GPU arm, OpenMP over "
+                     "sequences on %d threads; static build, prefill and warm-up steps untimed" % (K, B, units, threads)}
+    # one thread, on as many of the same steps as fit the budget
+    per_step_s = dt * threads / max(K, 1)
+    K1 = int(max(1, min(K, single_thread_budget_s / max(per_step_s, 1e-9))))
+    ob = fresh()
+    c0 = ob.counters()
+    t3 = time.perf_counter()
+    ob.run(new_tokens[Wm:Wm + K1], counts[Wm:Wm + K1], L, 1)
+    dt1 = time.perf_counter() - t3
+    u1 = ob.counters()["seq_steps"] - c0["seq_steps"]
+    ob.close()
+    res["single_thread_value"] = u1 / dt1
+    res["single_thread_sample"] = "the first %d of those steps" % K1
+    return res
 
+
+def _oracle_child(conn, name, batch, corpus_tokens, Wm, K, threads):
+    try:
+        base = variant(name, batch, corpus_tokens)
+        res = oracle_leg(base, Wm, K, threads, ready=lambda info: conn.send(("ready", info)),
+                         wait_for_go=lambda: conn.recv())
+        conn.send(("done", res))
+    except BaseException as ex:                          # the parent reports why there is no baseline
+        try:
+            conn.send(("error", "%s: %s" % (type(ex).__name__, ex)))
+        except Exception:
+            pass
+    finally:
+        conn.close()
+
+
+class OracleChildren:
+    """One child process per workload, started (spawn) before the first CUDA call."""
+
+    def __init__(self, names, args, Wm):
+        import multiprocessing as mp
+        self.ctx = mp.get_context("spawn")
+        self.kids = {}
+        self.threads = os.cpu_count() or 1
+        for name in names:
+            batch = args.batch if name == args.workload else 0
+            ctok = args.corpus_tokens if name == args.workload else 0
+            need_gb = estimate_oracle_gb(variant(name, batch, ctok))
+            avail = mem_available_gb()
+            if avail is not None and avail < need_gb + 24:
+                self.kids[name] = ("unavailable", "host has %.0f GB available, the oracle's automaton needs about %.0f GB"
+                                   % (avail, need_gb))
+                continue
+            parent, child = self.ctx.Pipe()
+            p = self.ctx.Process(target=_oracle_child, args=(child, name, batch, ctok, Wm, args.steps, self.threads),
+                                 daemon=True)
+            p.start()
+            child.close()
+            self.kids[name] = (p, parent)
+
+    def collect(self, name, wait_s):
+        """Let `name`'s child run its timed part now (nothing else is running) and return its result."""
+        kid = self.kids.get(name)
+        if kid is None:
+            return {"unavailable": "not requested"}
+        if kid[0] == "unavailable":
+            return {"unavailable": kid[1]}
+        p, conn = kid
+        try:
+            if not conn.poll(wait_s):
+                p.terminate()
+                return {"unavailable": "the oracle's automaton was not built within %d s" % wait_s}
+            tag, info = conn.recv()
+            if tag != "ready":
+                return {"unavailable": str(info)}
+            conn.send("go")
+            if not conn.poll(600):
+                p.terminate()
+                return {"unavailable": "the oracle's timed run did not end within 600 s"}
+            tag, res = conn.recv()
+            p.join(timeout=30)
+            return res if tag == "done" else {"unavailable": str(res)}
+        except (EOFError, OSError) as ex:
+            return {"unavailable": "oracle process ended early (%s)" % ex}
+
+    def close(self):
+        for kid in self.kids.values():
+            if kid[0] != "unavailable" and kid[0].is_alive():
+                kid[0].terminate()
+
+
+def mem_available_gb():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) / 1e6
+    except OSError:
+        pass
+    return None
+
+
+def estimate_oracle_gb(base: W.Spec) -> float:
+    """Host memory of the oracle's static automaton (about 1.3 states and 2.1 transitions per corpus
+    token, one small heap block per state) plus the corpus and the sequences' own automata."""
+    n = base.corpus_len
+    return (n * 1.3 * (29 + 32) + n * 4 * 2 + base.batch * (base.prompt_len + base.gen_len) * 200) / 1e9
+
+
+# ---------------------------------------------------------------------------------------------
+# the GPU arm
+# ---------------------------------------------------------------------------------------------
 
 def tree_draft_timing(P, st, batch, prepare, out, flush):
     """Time sam_tree_draft (best-first tree over the top-k successors, Algorithm 5) from the static states
@@ -244,51 +455,24 @@ def closed_loop(P, batch, seqs, spec, L):
             "note": "target = the sequence's own continuation (synthetic); torch gathers the target rows"}
 
 
-def main_reference(args):
-    rank, world, _ = dist_env()
-    if rank != 0:
-        return 0
-    spec = W.SPECS[args.workload]
-    corpus = W.make_corpus(spec)
-    seqs, counts, new_tokens = W.make_sequences(spec, corpus)
-    K = min(args.steps, counts.shape[0] - args.warmup)
-    threads = os.cpu_count() or 1
-    dt, units, drafts, _ = run_oracle_timed(spec, corpus, seqs, counts, new_tokens, args.warmup, args.warmup + K, threads)
-    value = units / dt
-    line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": K, "warmup": args.warmup, "ms_per_step": dt * 1e3 / K, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": spec.name, "batch": spec.batch, "prompt_len": spec.prompt_len,
-                   "gen_len": spec.gen_len, "draft_len": spec.draft_len, "corpus_tokens": spec.corpus_len},
-        "draft_tokens_per_sec": drafts / dt,
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                         "sample": "decoding steps [%d, %d) of %s, all %d sequences, OpenMP over sequences; "
-                                   "static build and prefill untimed" % (args.warmup, args.warmup + K, spec.name, spec.batch)},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0,
-    }
-    print(json.dumps(line))
-    return 0
+def peak_stream():
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        return float(peaks["hbm_gbs"]), "measured stream copy"
+    except Exception:
+        return 6650.0, "fallback stream copy"
 
 
-def main_ours(args):
+def measure_gpu(P, args, name, rank, world, local_rank, full):
+    """One workload on this rank's GPU.  `full`: the headline treatment (graph replay, probes, clock samples)."""
     import torch
-    rank, world, local_rank = dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the retrieval path has no CPU implementation")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
-    import paper_2411_10666_b200 as P
     sd = P.binding
-    P.lib()
-
-    base = W.SPECS[args.workload]
-    if args.batch > 0:
-        base = W.scaled(base, batch=args.batch)
+    is_named = name == args.workload
+    base = variant(name, args.batch if is_named else 0, args.corpus_tokens if is_named else 0)
+    label = workload_label(name, args.batch if is_named else 0, args.corpus_tokens if is_named else 0)
+    t0 = time.perf_counter()
     spec, corpus, seqs, counts, new_tokens = shard_workload(base, rank, world)
+    inputs_s = time.perf_counter() - t0
     B, L = seqs.shape[0], spec.draft_len
     msl = spec.prompt_len + spec.gen_len
     Wm = args.warmup
@@ -296,15 +480,19 @@ def main_ours(args):
     assert K >= 1 and Wm >= 3, "need at least 3 warm-up steps and 1 timed step"
 
     t0 = time.perf_counter()
-    st = P.StaticSam.build(corpus, spec.vocab, device=local_rank, tree_topk=4 if args.tree_draft else 0)
+    topk = 4 if (args.tree_draft and full) else 0
+    if args.cache_dir and rank == 0:
+        st, static_source = P.StaticSam.cached(corpus, spec.vocab, args.cache_dir, device=local_rank, tree_topk=topk)
+    else:
+        st, static_source = P.StaticSam.build(corpus, spec.vocab, device=local_rank, tree_topk=topk), "built"
     build_s = time.perf_counter() - t0
     info = st.info
     batch = P.Batch(st, B, msl, max_draft_len=L, max_host_stride=spec.accept_max)
     dev = batch.device
     prompts = torch.from_numpy(np.ascontiguousarray(seqs[:, :spec.prompt_len])).to(dev)
     pcount = torch.full((B,), spec.prompt_len, dtype=torch.int32, device=dev)
-    nt_dev = torch.from_numpy(new_tokens).to(dev)
-    ct_dev = torch.from_numpy(counts).to(dev)
+    nt_dev = torch.from_numpy(new_tokens[:Wm + K]).to(dev)
+    ct_dev = torch.from_numpy(counts[:Wm + K]).to(dev)
     out = P.StepOutputs(B, L, dev)
     flush = torch.empty(288 << 20, dtype=torch.uint8, device=dev)      # larger than the 126 MB L2
 
@@ -326,12 +514,15 @@ def main_ours(args):
     torch.cuda.synchronize()
     prefill_ms = e0.elapsed_time(e1)
 
-    gpu_id = str(torch.cuda.current_device())
-    try:                                                  # the physical GPU, whatever CUDA_VISIBLE_DEVICES says
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
-    except Exception:
-        pass
-    sampler = ClockSampler(gpu_id) if rank == 0 else None
+    sampler = None
+    if full and rank == 0:
+        gpu_id = str(torch.cuda.current_device())
+        try:                                              # the physical GPU, whatever CUDA_VISIBLE_DEVICES says
+            gpu_id = "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+        except Exception:
+            pass
+        sampler = ClockSampler(gpu_id)
+    min_seconds = args.min_seconds if full else min(args.min_seconds, 1.0)
     times = []
     t_start = time.perf_counter()
     while True:
@@ -347,7 +538,7 @@ def main_ours(args):
             torch.distributed.barrier()
         times.append(e0.elapsed_time(e1))
         elapsed = time.perf_counter() - t_start
-        stop = len(times) >= 3 and (elapsed >= args.min_seconds or len(times) >= args.max_repeats)
+        stop = len(times) >= 3 and (elapsed >= min_seconds or len(times) >= args.max_repeats)
         if world > 1:                                                   # all ranks stop together
             flag = torch.tensor([1 if stop else 0], device=dev)
             torch.distributed.all_reduce(flag, op=torch.distributed.ReduceOp.MAX)
@@ -359,7 +550,7 @@ def main_ours(args):
     # the same K launches captured once in a CUDA graph and replayed (reported beside the headline,
     # which stays the plain stream launches)
     graph_ms = None
-    if world == 1:
+    if world == 1 and full:
         try:
             side = torch.cuda.Stream()
             prepare()
@@ -379,13 +570,12 @@ def main_ours(args):
                 gt.append(e0.elapsed_time(e1))
             graph_ms = statistics.median(gt)
             del graph
-        except Exception as ex:                                   # capture unsupported: report why
+        except Exception:                                         # capture unsupported: no figure
             graph_ms = None
-            graph_err = str(ex)
 
     # end to end through the host-array call: pinned inputs, H2D + step + D2H + sync every step
-    nt_pin = torch.from_numpy(new_tokens).pin_memory()
-    ct_pin = torch.from_numpy(counts).pin_memory()
+    nt_pin = torch.from_numpy(new_tokens[:Wm + K]).pin_memory()
+    ct_pin = torch.from_numpy(counts[:Wm + K]).pin_memory()
     mk = lambda *s: torch.empty(s, dtype=torch.int32).pin_memory()
     ho = [mk(B, L), mk(B), mk(B, 2), mk(B), mk(B, 2), mk(B)]
     ho_ptr = [t.data_ptr() for t in ho]                     # addresses are passed as plain ints
@@ -412,33 +602,35 @@ def main_ours(args):
     draft_tokens = int((per.draft_len * active).sum().item())
     accepted_tokens = int(counts[Wm:Wm + K].sum())
     torch.cuda.synchronize()
+    del per
 
     ms_local = statistics.median(times)
     ms, units_all = reduce_max_sum(ms_local, units, world)
     e2e_ms, _ = reduce_max_sum(statistics.median(e2e_times), units, world)
     _, drafts_all = reduce_max_sum(0.0, draft_tokens, world)
-    if rank != 0:
-        if world > 1:
-            torch.distributed.destroy_process_group()
-        return 0
 
-    value = units_all / (ms * 1e-3)
     launch_us = ms_local * 1e3 / K
-    algo_b = ALGO_BYTES[base.name]
-    achieved = algo_b * (units / K) / (launch_us * 1e-6) / 1e9          # GB/s of one launch on this rank
-    peak_src = "fallback"
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-        peak, peak_src = float(peaks["hbm_gbs"]), "measured"
-    except Exception:
-        peak = 6650.0
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(base.name) if args.batch <= 0 else None, "peak_source": peak_src + " stream copy",
-                "kernel": "sam_step_kernel", "launch_us": launch_us,
-                "algorithmic_bytes_per_sequence_step": algo_b,
-                "sequence_steps_per_launch": units / K}
+    res = {
+        "label": label, "base": base, "K": K, "Wm": Wm, "B": B, "L": L, "world": world,
+        "value": units_all / (ms * 1e-3), "ms_per_step": ms / K, "launch_us": launch_us,
+        "units_local": units, "units_all": units_all,
+        "draft_tokens_per_sec": drafts_all / (ms * 1e-3),
+        "accepted_tokens_per_sec": accepted_tokens * world / (ms * 1e-3),
+        "best_ms_per_step": min(times) / K, "repeats": len(times),
+        "prefill_tokens_per_sec": B * spec.prompt_len / (prefill_ms * 1e-3),
+        "static": {"states": int(info.n_states), "transitions": int(info.n_transitions), "device_bytes": int(info.device_bytes),
+                   "seconds": build_s, "source": static_source, "inputs_seconds": inputs_s},
+        "status_all_ok": status_ok,
+        "e2e": {"value": units_all / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": B * spec.accept_max * 4 + B * 4, "d2h_bytes_per_step": B * (L + 7) * 4,
+                "ms_per_step": e2e_ms / K, "api": "sam_step_host"},
+        "gpu_launches": K * batch.launches_per_step(), "launches_per_step": batch.launches_per_step(),
+        "graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms / K, "value": units / (graph_ms * 1e-3),
+                                                       "note": "the K sam_step launches captured in one CUDA graph"},
+        "clocks": clocks,
+    }
 
-    if not args.no_probes:
+    if full and rank == 0 and not args.no_probes:
         # the random-access denominators, measured now on a buffer the size of the static store
         fp = min(max(int(info.device_bytes), 256 << 20), 8 << 30)
         buf = torch.empty(fp, dtype=torch.uint8, device=dev)
@@ -446,55 +638,190 @@ def main_ours(args):
         for g in (32, 64, 128):
             gbps, mreq = sd.sam_probe_random_read(buf, g, iters=3)
             rnd[str(g)] = {"GB/s": round(gbps, 1), "Mreq/s": round(mreq, 1)}
-        chains = 2 * B
+        chains = min(2 * B, 65536)
         ns1 = sd.sam_probe_chase(buf, 20000, chains=1)
         nsc = sd.sam_probe_chase(buf, 20000, chains=chains)
         del buf
-        roofline["random_read"] = rnd
-        roofline["frac_of_random_32B"] = achieved / rnd["32"]["GB/s"]
-        roofline["dependent_load_ns"] = {"1_chain": round(ns1, 1), "%d_chains" % chains: round(nsc, 1)}
+        res["probes"] = {"random_read": rnd, "footprint_bytes": fp,
+                         "dependent_load_ns": {"1_chain": round(ns1, 1), "%d_chains" % chains: round(nsc, 1)},
+                         "chains": chains}
+    if full and args.tree_draft:
+        res["tree_draft"] = tree_draft_timing(P, st, batch, prepare, out, flush)
+    if full and args.closed_loop:
+        res["closed_loop"] = closed_loop(P, batch, seqs, spec, L)
 
+    batch.close()
+    st.close()
+    del batch, st, flush, nt_dev, ct_dev, prompts, out, nt_pin, ct_pin, ho
+    torch.cuda.empty_cache()
+    return res
+
+
+def roofline_block(res, cpu, probes):
+    """The roofline object of one workload: algorithmic bytes per launch over the launch time against
+    the stream-copy peak, the random-read rate and the dependent-access bound beside it."""
+    name = res["base"].name
+    L = res["L"]
+    counters = cpu.get("counters") if cpu else None
+    if counters and res["world"] == 1:
+        ab = algorithmic_bytes(counters, L)
+        algo_b, algo_src = ab["total"], "CPU oracle's operation counters over exactly the timed steps"
+    else:
+        ab = None
+        algo_b, algo_src = ALGO_BYTES_WHOLE_PHASE[name], "CPU oracle's operation counters averaged over the recipe's whole generation phase"
+    per_launch = res["units_local"] / res["K"]
+    achieved = algo_b * per_launch / (res["launch_us"] * 1e-6) / 1e9
+    peak, peak_src = peak_stream()
+    digest = kernel_digest()
+    cap = NCU_TRAFFIC.get(res["label"])
+    traffic, traffic_src = None, "no ncu capture of this workload with the kernel sources as they stand (digest %s)" % digest
+    if cap is not None:
+        if cap[2] == digest:
+            traffic = cap[0] * (per_launch / cap[1]) if cap[1] else cap[0]
+            traffic_src = cap[3]
+        else:
+            traffic_src = "ncu capture is of kernel sources %s, they are now %s: not reported" % (cap[2], digest)
+    r = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+         "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src,
+         "kernel": "sam_step_kernel", "launch_us": res["launch_us"],
+         "algorithmic_bytes_per_sequence_step": algo_b, "algorithmic_bytes_source": algo_src,
+         "sequence_steps_per_launch": per_launch}
+    if ab:
+        r["algorithmic_bytes_split"] = {k: round(v, 1) for k, v in ab.items()}
+    if probes:
+        r["random_read"] = probes["random_read"]
+        r["frac_of_random_32B"] = achieved / probes["random_read"]["32"]["GB/s"]
+        r["dependent_load_ns"] = probes["dependent_load_ns"]
+        if counters:
+            # the dependent-access bound: a sequence's two chains run side by side, each makes its
+            # accesses one after the other, so a sequence-step takes at least (accesses of the longer
+            # chain) x (latency of a dependent load at this concurrency)
+            d = dependent_accesses(counters)
+            t_dep = probes["dependent_load_ns"]["%d_chains" % probes["chains"]] * 1e-9
+            dmax = max(d.values())
+            bound = res["B"] / (dmax * t_dep)
+            r["concurrency_bound"] = {"value": bound, "unit": UNIT,
+                                      "formula": "B / (d x t_dep): B sequences in flight, d dependent accesses of the longer chain per sequence-step, t_dep at 2B chains",
+                                      "dependent_accesses_per_sequence_step": {k: round(v, 2) for k, v in d.items()},
+                                      "note": "d counts the accesses Algorithms 1 and 3 make one after the other; the kernel reads guessed states side by side where it can, so it may exceed this figure"}
+            r["frac_of_concurrency_bound"] = (res["units_local"] / (res["launch_us"] * 1e-6 * res["K"])) / bound
+    return r
+
+
+def main_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    base = variant(args.workload, args.batch, args.corpus_tokens)
+    label = workload_label(args.workload, args.batch, args.corpus_tokens)
+    threads = os.cpu_count() or 1
+    res = oracle_leg(base, args.warmup, args.steps, threads)
+    K = res["steps"]
+    value = res["value"]
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32", "data": "synthetic",
-        "config": {"workload": base.name + ("" if args.batch <= 0 else " (recipe run with %d sequences)" % args.batch), "batch_per_gpu": B, "global_batch": B * world,
-                   "prompt_len": spec.prompt_len, "gen_len": spec.gen_len, "draft_len": L,
-                   "corpus_tokens": spec.corpus_len, "vocab": spec.vocab,
-                   "static_states": int(info.n_states), "static_bytes": int(info.device_bytes),
-                   "parallelism": "batch-sharded x%d, static automaton replicated" % world,
-                   "l2": "L2 flushed (288 MB write) before each timed region; static store %.2f GB exceeds the 126 MB L2; "
-                         "per-sequence automata stay cache-warm between consecutive steps" % (info.device_bytes / 1e9),
-                   "repeats": len(times), "timing": "median of repeats, CUDA events, max over ranks"},
-        "draft_tokens_per_sec": drafts_all / (ms * 1e-3),
-        "accepted_tokens_per_sec": accepted_tokens * world / (ms * 1e-3),
-        "best_ms_per_step": min(times) / K,
-        "prefill_tokens_per_sec": B * spec.prompt_len / (prefill_ms * 1e-3),
-        "static_build_seconds": build_s,
-        "status_all_ok": status_ok,
-        "e2e": {"value": units_all / (e2e_ms * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": B * spec.accept_max * 4 + B * 4, "d2h_bytes_per_step": B * (L + 7) * 4,
-                "ms_per_step": e2e_ms / K, "api": "sam_step_host"},
-        "gpu_launches": K * batch.launches_per_step(),
-        "graph_replay": None if graph_ms is None else {"ms_per_step": graph_ms / K, "value": units / (graph_ms * 1e-3),
-                                                       "note": "the K sam_step launches captured in one CUDA graph"},
-        "clocks": clocks,
-        "roofline": roofline,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": K, "warmup": args.warmup, "ms_per_step": res["seconds"] * 1e3 / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": config_dict(base, label, world),
+        "draft_tokens_per_sec": res["draft_tokens_per_sec"],
+        "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample", "single_thread_value",
+                                             "single_thread_sample", "oracle_build_seconds")},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
     }
+    print(json.dumps(line))
+    return 0
 
-    if args.tree_draft:
-        line["tree_draft"] = tree_draft_timing(P, st, batch, prepare, out, flush)
-    if args.closed_loop:
-        line["closed_loop"] = closed_loop(P, batch, seqs, spec, L)
 
-    if world == 1 and not args.no_cpu_baseline:
-        cores = os.cpu_count() or 1
-        dt, u, _, S = run_oracle_timed(base, corpus, seqs, counts, new_tokens, Wm, Wm + K, cores)
-        dt1, u1, _, _ = run_oracle_timed(base, corpus, seqs, counts, new_tokens, Wm, Wm + K, 1, static=S)
-        line["cpu_baseline"] = {"value": u / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "single_thread_value": u1 / dt1,
-                                "sample": "the same %d decoding steps x %d sequences (%d sequence-steps), OpenMP over "
-                                          "sequences; static build and prefill untimed" % (K, B, u)}
+def main_ours(args):
+    rank, world, local_rank = dist_env()
+    one = world == 1
+    names = [args.workload]
+    if one and not args.no_all_workloads and not args.batch and not args.corpus_tokens:
+        names += [n for n in ORDER if n != args.workload]
+    kids = None
+    if one and not args.no_cpu_baseline:
+        kids = OracleChildren(names, args, args.warmup)       # spawned before the first CUDA call
+
+    import torch
+    if not torch.cuda.is_available():
+        if kids:
+            kids.close()
+        raise SystemExit("bench.py needs a CUDA device: the retrieval path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+    import paper_2411_10666_b200 as P
+    P.lib()
+
+    t_all = time.perf_counter()
+    results = {}
+    for n in names:
+        results[n] = measure_gpu(P, args, n, rank, world, local_rank, full=(n == args.workload))
+    gpu_part_s = time.perf_counter() - t_all
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return 0
+
+    # the oracle's timed runs, one after the other, smallest automaton first (the largest is still building)
+    cpu = {}
+    if kids:
+        t_wait = time.perf_counter()
+        for n in sorted(names, key=lambda n: variant(n).corpus_len if n != args.workload else 1 << 62):
+            left = max(30.0, args.cpu_wait_seconds - (time.perf_counter() - t_wait))
+            cpu[n] = kids.collect(n, left)
+        kids.close()
+
+    head = results[args.workload]
+    probes = head.get("probes")
+    head_cpu = cpu.get(args.workload)
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": head["K"], "warmup": head["Wm"],
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": config_dict(head["base"], head["label"], world),
+        "timing": {"repeats": head["repeats"], "how": "median of repeats, CUDA events, max over ranks",
+                   "gpu_part_seconds": gpu_part_s},
+        "draft_tokens_per_sec": head["draft_tokens_per_sec"],
+        "accepted_tokens_per_sec": head["accepted_tokens_per_sec"],
+        "best_ms_per_step": head["best_ms_per_step"],
+        "prefill_tokens_per_sec": head["prefill_tokens_per_sec"],
+        "static": head["static"], "static_build_seconds": head["static"]["seconds"],
+        "status_all_ok": head["status_all_ok"],
+        "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "graph_replay": head["graph_replay"],
+        "clocks": head["clocks"],
+        "roofline": roofline_block(head, head_cpu if head_cpu and "value" in head_cpu else None, probes),
+    }
+    for k in ("tree_draft", "closed_loop"):
+        if k in head:
+            line[k] = head[k]
+    if head_cpu is not None:
+        line["cpu_baseline"] = ({k: v for k, v in head_cpu.items() if k != "counters"} if "value" in head_cpu
+                                else {"value": None, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                      "sample": "none", "unavailable": head_cpu.get("unavailable")})
+    if len(names) > 1:
+        allw = {}
+        for n in ORDER:
+            r = results[n]
+            c = cpu.get(n)
+            ok = bool(c) and "value" in c
+            rf = roofline_block(r, c if ok else None, probes if n == args.workload else None)
+            allw[n] = {"value": r["value"], "unit": UNIT, "us_per_step": r["ms_per_step"] * 1e3, "batch": r["B"],
+                       "steps": r["K"], "repeats": r["repeats"], "launches_per_step": r["launches_per_step"],
+                       "draft_tokens_per_sec": r["draft_tokens_per_sec"], "e2e_value": r["e2e"]["value"],
+                       "static_bytes": r["static"]["device_bytes"], "status_all_ok": r["status_all_ok"],
+                       "algorithmic_bytes_per_sequence_step": rf["algorithmic_bytes_per_sequence_step"],
+                       "achieved_GBps": rf["achieved"], "frac_of_stream_copy": rf["frac"],
+                       "cpu_oracle_value": c["value"] if ok else None,
+                       "cpu_oracle_cores": c["cores"] if ok else None,
+                       "cpu_oracle_note": None if ok else (c or {}).get("unavailable", "not run")}
+            if probes:
+                allw[n]["frac_of_random_32B"] = rf["achieved"] / probes["random_read"]["32"]["GB/s"]
+        line["all_workloads"] = allw
+        line["all_workloads_note"] = ("the four other recipes measured the same way with a shorter timed region; the random-read "
+                                      "rate in their fractions is the one measured over the headline workload's footprint")
     print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()

@@ -378,6 +378,19 @@ def sam_probe_chase(buf, hops: int, chains: int = 1, stream=None):
 # small owner objects (lifetime + torch memory), still no arithmetic
 # ---------------------------------------------------------------------------------------------
 
+def _on_ram_disk(path: str) -> bool:
+    """True if `path` lies on a memory-backed filesystem (an image written there would use up RAM)."""
+    try:
+        real, best, kind = os.path.realpath(path), "", ""
+        for line in open("/proc/mounts"):
+            f = line.split()
+            if len(f) >= 3 and (real == f[1] or real.startswith(f[1].rstrip("/") + "/")) and len(f[1]) >= len(best):
+                best, kind = f[1], f[2]
+        return kind in ("tmpfs", "ramfs")
+    except OSError:
+        return False
+
+
 class StaticSam:
     """A static automaton on a device.  `StaticSam.build(corpus, vocab)` or `StaticSam.load(path)`."""
 
@@ -394,6 +407,36 @@ class StaticSam:
 
     def save(self, path: str):
         sam_static_save(self.handle, path)
+
+    @classmethod
+    def cached(cls, corpus, vocab: int, cache_dir: str, device: int = 0, tree_topk: int = 0):
+        """The automaton of `corpus` from a saved image under `cache_dir` when there is one, else built
+        and, room on the disk permitting, saved there.  The file name is a digest of the corpus bytes,
+        the vocabulary, the top-k setting and the library version, so a stale image is never picked up;
+        an image that fails its checksum is rebuilt.  Returns (automaton, "loaded" | "built")."""
+        import hashlib
+        import shutil
+        c = _np32(corpus)
+        h = hashlib.blake2b(digest_size=12)
+        h.update(memoryview(c).cast("B"))
+        h.update(("|%d|%d|%s" % (vocab, tree_topk, lib().sam_version().decode())).encode())
+        path = os.path.join(cache_dir, "static-%s.samimg" % h.hexdigest())
+        if os.path.exists(path):
+            try:
+                return cls.load(path, device), "loaded"
+            except SamError:
+                pass
+        st = cls.build(c, vocab, device, 0.0, tree_topk)
+        try:
+            os.makedirs(cache_dir, exist_ok=True)
+            need = int(st.info.device_bytes * 1.1) + (2 << 30)
+            if not _on_ram_disk(cache_dir) and shutil.disk_usage(cache_dir).free > need:
+                tmp = path + ".tmp%d" % os.getpid()
+                st.save(tmp)
+                os.replace(tmp, path)
+        except (OSError, SamError):
+            pass                                        # a cache that cannot be written is not an error
+        return st, "built"
 
     @property
     def info(self) -> StaticInfo:

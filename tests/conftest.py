@@ -8,4 +8,3 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (the parity tests proper)")
-    config.addinivalue_line("markers", "full: full-size workloads that take minutes (opt in with SAMDRAFT_FULL=1)")

@@ -227,7 +227,8 @@ def test_static_matches_in_prefix_states(P):
             ref, ob, _ = oracle_run(corpus, vocab, empty, nt, ct, L, n, stop_token=stop)
             got, batch = gpu_run(P, st, vocab, empty, nt, ct, L, n, stop_token=stop)
             assert_same(got, ref, "vocab %d N %d L %d" % (vocab, N, L))
-            assert (got["source"] == 1).any()
+            assert got["match_len"][:, :, 0].max() >= min(N, 8)
+            assert N < 200 or (got["source"] == 1).any()      # in the short periodic corpora the own text ties or wins
 
 
 def test_large_batch_is_ordered_by_token_count(P):
@@ -299,16 +300,58 @@ def test_c2_full_size_bench_configuration(P):
             assert (got["draft_tokens"][s + 1, b, :dl] == w.corpus[e1:e1 + dl]).all()
 
 
-@pytest.mark.skipif(os.environ.get("SAMDRAFT_FULL") != "1", reason="minutes and tens of GB: set SAMDRAFT_FULL=1")
+def _mem_available_gb():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) / 1e6
+    except OSError:
+        pass
+    return 1e9
+
+
+# host memory (GB) the two independent automata of a full-size case need side by side, with margin
+FULL_SIZE_HOST_GB = {"c4": 4, "c3": 60, "c5": 110}
+
+
 @pytest.mark.parametrize("key", ["c4", "c3", "c5"])
 def test_full_size_configs(P, key):
+    """The recipe at its full size, launched as the benchmark launches it (prefill step, then every
+    decoding step through sam_run_steps; the slot-ordering launch included for c5): every output of
+    every step equals the oracle's, and the library's static automaton has the oracle's number of
+    states and transitions.  The oracle's automaton is built in a thread while the library builds its
+    own and the GPU runs.  Skipped only when the host cannot hold both automata."""
+    import threading
+    import torch
+    avail = _mem_available_gb()
+    free_dev = torch.cuda.mem_get_info()[0] / 1e9
+    if avail < FULL_SIZE_HOST_GB[key]:
+        pytest.skip("host has %.0f GB available; %s at full size needs about %d GB" % (avail, key, FULL_SIZE_HOST_GB[key]))
     spec = W.SPECS[key]
+    if free_dev < spec.corpus_len * 100e-9 + 6:
+        pytest.skip("device has %.0f GB free; %s at full size needs about %.0f GB" % (free_dev, key, spec.corpus_len * 100e-9 + 6))
     w = W.make(spec)
     L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    box = {}
+
+    def build_oracle():
+        try:
+            box["S"] = oracle.Sam(w.corpus)
+        except BaseException as ex:                     # re-raised in the test's own thread
+            box["err"] = ex
+
+    th = threading.Thread(target=build_oracle)
+    th.start()
     st = P.StaticSam.build(w.corpus, spec.vocab)
     got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
-    ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=os.cpu_count())
+    assert batch.launches_per_step() == (2 if spec.batch >= 1536 else 1)
+    th.join()
+    if "err" in box:
+        raise box["err"]
+    ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, static=box["S"],
+                            threads=os.cpu_count())
     assert_same(got, ref, key)
+    assert (got["status"] == 0).all()
     assert st.info.n_states == S.n_states and st.info.n_transitions == S.n_transitions
 
 
