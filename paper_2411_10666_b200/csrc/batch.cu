@@ -53,7 +53,7 @@ int plan(const sam_batch_opts_t* o, WsLayout* w) {
     w->off_free = off;  off = sam_align_up(off + (size_t)slabs * 4, 256);
     w->off_owner = off; off = sam_align_up(off + (size_t)slabs * 4, 256);
     w->off_reset = off; off = sam_align_up(off + (size_t)o->batch * 4 * 2, 256);   // flags + slot list
-    w->off_order = off; off = sam_align_up(off + (size_t)o->batch * 4 * 3, 256);   // two order buffers + the sort keys
+    w->off_order = off; off = sam_align_up(off + (size_t)o->batch * 4 * 3 + 64, 256);   // two order buffers, the sort keys, two counts
     w->off_text = off;  off = sam_align_up(off + (size_t)o->batch * w->text_stride * 4, 256);
     w->off_pstate = off; off = sam_align_up(off + (size_t)o->batch * w->text_stride * 4, 256);
     w->off_root = off;  off = sam_align_up(off + (size_t)o->batch * w->root_cap * 8, 256);

@@ -64,7 +64,10 @@
 // control-block word indices
 enum {
     CB_STATUS = 0, CB_NTOK, CB_NSTATES, CB_LAST, CB_S1, CB_L1, CB_S2, CB_L2,
-    CB_S1FLAG, CB_BLK_CUR, CB_BLK_END, CB_NRECSLABS, CB_ROOTDEG, CB_RSV13, CB_RSV14, CB_RSV15,
+    CB_S1FLAG, CB_BLK_CUR, CB_BLK_END, CB_NRECSLABS, CB_ROOTDEG,
+    CB_ARRIVE,        // split step: how many of the slot's two sides have finished (parity: 2 per step)
+    CB_NTOK_S,        // the text length as the static side keeps it (it may not read CB_NTOK while the dynamic side writes it)
+    CB_ERR_S,         // split step: error met by the static side (walk limit), 0 otherwise
     CB_SLABTAB = 16,  // .. 47
     CB_REC1 = 48,     // .. 55: copy of the static match state's record (valid when s1 != 0)
     CB_REC2 = 56      // .. 63: copy of the dynamic match state's record (valid when s2 != 0)
@@ -124,7 +127,7 @@ struct SamBatchView {
     int32_t* free_stack;      // [pool_slabs]
     int32_t* slab_owner;      // [pool_slabs], -1 = free
     int32_t* reset_flag;      // [B]
-    int32_t* order;           // [3][B]: slots sorted by their step's token count (large batches), two buffers in turn; then the sort keys
+    int32_t* order;           // [3][B] + 16: slots sorted by their step's token count (large batches), two buffers in turn; the sort keys; per buffer, at 3B + 8 x buffer, the number of slots with many tokens
     int32_t* text;            // [B][text_stride]
     uint32_t* pstate;         // [B][text_stride]: id of the state created by each text position
     uint2* root_tab;          // [B][root_cap]

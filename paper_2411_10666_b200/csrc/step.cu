@@ -54,12 +54,19 @@ struct StepArgs {
     int32_t* v_counts_out; int32_t* v_accepted_out;
     // optional: block i works on slot order[i] (slots with many tokens first; see order_slots_kernel)
     const int32_t* order;
+    // split step (sam_step_split_kernel): blocks [0, n_warp_blocks) run the static side of one slot each (the
+    // first *split_count slots of `order`, those with many tokens), the next n_lane_blocks blocks the static
+    // side of 32 slots each, the remaining blocks the dynamic side of one slot each
+    int32_t n_warp_blocks, n_lane_blocks;
+    const int32_t* split_count;
 };
 
 // ------------------------------------------------------------------ draft read
 // d[r] (lane j of round r) = text[e + 32 r + j] for 32 r + j < dl, else -1.  The window is read as
 // aligned 16-byte vectors (nine lanes per 32 tokens) and realigned with shuffles.
-template <bool READONLY>
+// READ: 0 plain loads, 1 read-only path (text that no kernel writes), 2 loads that bypass the L1 (text
+// written by another block of the grid that is running).
+template <int READ>
 __device__ __forceinline__ void gather_draft(const int32_t* text, int64_t e, int dl, int L, int lane,
                                              int32_t d[MAX_DRAFT_REGS]) {
     const int off = (int)(e & 3);
@@ -72,7 +79,7 @@ __device__ __forceinline__ void gather_draft(const int32_t* text, int64_t e, int
         if (r * 32 < L) {
             int4 q = make_int4(0, 0, 0, 0);
             const int vi = 8 * r + lane;
-            if (lane < 9 && vi < nvec) q = READONLY ? __ldg(v + vi) : v[vi];
+            if (lane < 9 && vi < nvec) q = READ == 1 ? __ldg(v + vi) : READ == 2 ? __ldcg(v + vi) : v[vi];
             int x0 = __shfl_sync(FULL, q.x, src), x1 = __shfl_sync(FULL, q.y, src);
             int x2 = __shfl_sync(FULL, q.z, src), x3 = __shfl_sync(FULL, q.w, src);
             int val = comp == 0 ? x0 : comp == 1 ? x1 : comp == 2 ? x2 : x3;
@@ -691,6 +698,203 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
     return r;
 }
 
+// The static side of one slot's step, run by one warp: Transfer (Algorithm 1) for each of the slot's m
+// tokens, then the static words of the control block.  cw holds control words 0..31 as read at the start
+// of the step; on entry (ra, rb) is the copy of the match state's record kept in the control block, ntok0
+// the text length before the step.  On exit (s, sf, l) is the match state, and, if l > 0 and no error,
+// (ra, rb) its record.  DRAFT: also fetch the draft after the state's first end position into d / my_dl
+// (requested early where the address is known early).
+template <bool DRAFT>
+__device__ __forceinline__ void static_chain(const StepArgs& A, int lane, uint32_t* cb, uint32_t cw, int32_t tok_first,
+                                             const int32_t* toks, int m, uint32_t ntok0, uint4& ra, uint4& rb,
+                                             uint32_t& s_out, uint32_t& sf_out, int32_t& l_out, int& err,
+                                             int32_t d[MAX_DRAFT_REGS], int32_t& my_dl) {
+    const int L = A.L;
+    uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
+    int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
+    bool have = s != 0;
+    // The match state is the state Build-SAM created for a whole corpus prefix (len == min_endpos:
+    // not a clone), the prefix ending at e.  Its transition on the next corpus token was created
+    // solid (len + 1) and a solid transition is never redirected, so it still leads to the state of
+    // the prefix one longer, with match length l + 1.  The state may occur more than once and have
+    // other transitions too ("ab" in "ababc"): nothing is assumed about those.  The step's tokens
+    // are compared with the corpus after e; as long as they agree the state is taken from the
+    // position -> state array, and the first token that differs goes through the ordinary Transfer
+    // below.  All in one round trip, in which the draft after e + m is requested as well in case
+    // every token agrees.
+    int j0 = 0;                      // tokens already taken
+    bool drafted = false;
+    if (have && m >= 1 && m <= 32 && ra.x == ra.z) {
+        const int64_t e = (int64_t)ra.z;
+        int32_t cx = -2; uint32_t px = 0;
+        if (lane < m && e + lane < A.S.n_tokens) { cx = __ldg(A.S.corpus + e + lane); px = __ldg(A.S.pstate + e + lane); }
+        const int64_t e2 = e + m;
+        const int64_t room = A.S.n_tokens - e2;
+        const int dl2 = (int)(room < L ? (room < 0 ? 0 : room) : L);
+        if (DRAFT) gather_draft<1>(A.S.corpus, e2, dl2, L, lane, d);
+        const unsigned agree = __ballot_sync(FULL, lane < m && cx == tok_first);
+        j0 = (~agree) ? __ffs(~agree) - 1 : 32;
+        if (j0 > 0) {
+            const uint32_t ref = __shfl_sync(FULL, px, j0 - 1);
+            s = ref & SAM_IDMASK; sf = ref >> 31; l += j0; have = false;
+            if (j0 == m) {                                  // the whole step: the draft is in already
+                ra = __ldg(A.S.rec + 2 * (size_t)s);        // its record, for the next step
+                rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
+                if (DRAFT) my_dl = cut_at_stop(d, dl2, lane, A.W.stop_token);
+                drafted = true;
+            }
+        }
+    }
+    for (int base = 0; base < m && !err && j0 < m; base += 32) {
+        const int i = base + lane;
+        uint32_t tk = 0, re = SAM_NONE;
+        if (i < m) { tk = (uint32_t)(base == 0 ? tok_first : toks[i]); re = __ldg(A.S.root_row + tk); }
+        const int cnt = min(32, m - base);
+        // Most tokens end a short match: the lookup misses, the link leads to the root, and the
+        // root row gives the next state u = root_row[t].  The token after that is then looked up
+        // in u — a lookup whose address is known now.  Lookups k = 0..7 (state root_row[t_k],
+        // token t_{k+1}) are read ahead here, eight lanes each: the state's record in lanes 0-1
+        // of the group, its hash bucket in all eight.  They are used if the matcher really is
+        // in that state when the token comes.
+        uint4 sp_rec[2], sp_ent[2];
+#pragma unroll
+        for (int r = 0; r < 2; r++) {
+            const int k = 4 * r + (lane >> 3), e = lane & 7;
+            const uint32_t uref = __shfl_sync(FULL, re, k);
+            const uint32_t tnext = __shfl_sync(FULL, tk, k + 1);
+            sp_rec[r] = make_uint4(0, 0, 0, 0);
+            sp_ent[r] = make_uint4(SAM_NONE, 0, 0, 0);
+            if (k + 1 < cnt && uref != SAM_NONE) {
+                const uint32_t u = uref & SAM_IDMASK;
+                if (e < 2) sp_rec[r] = __ldg(A.S.rec + 2 * (size_t)u + e);
+                if (uref >> 31)
+                    sp_ent[r] = __ldg(A.S.hash + (size_t)(sam_hash2(u, tnext) & A.S.hash_mask) * SAM_HASH_BUCKET + e);
+            }
+        }
+        for (int j = j0; j < cnt && !err; j++) {
+            bool pre = false;
+            uint4 pa = ra, pb = rb, pent = make_uint4(SAM_NONE, 0, 0, 0);
+            if (j >= 1 && j <= 8 && s != 0) {
+                const uint32_t prev = __shfl_sync(FULL, re, j - 1);
+                if (prev != SAM_NONE && (prev & SAM_IDMASK) == s) {        // the state read ahead
+                    const int k = j - 1, g8 = 8 * (k & 3);
+                    const uint4 xr = (k >> 2) ? sp_rec[1] : sp_rec[0];
+                    const uint4 xe = (k >> 2) ? sp_ent[1] : sp_ent[0];
+                    pa.x = __shfl_sync(FULL, xr.x, g8); pa.y = __shfl_sync(FULL, xr.y, g8);
+                    pa.z = __shfl_sync(FULL, xr.z, g8); pa.w = __shfl_sync(FULL, xr.w, g8);
+                    pb.x = __shfl_sync(FULL, xr.x, g8 + 1); pb.y = __shfl_sync(FULL, xr.y, g8 + 1);
+                    pb.z = __shfl_sync(FULL, xr.z, g8 + 1); pb.w = __shfl_sync(FULL, xr.w, g8 + 1);
+                    const int src = g8 + (lane & 7);
+                    pent.x = __shfl_sync(FULL, xe.x, src); pent.y = __shfl_sync(FULL, xe.y, src);
+                    pent.z = __shfl_sync(FULL, xe.z, src); pent.w = __shfl_sync(FULL, xe.w, src);
+                    pre = true;
+                }
+            }
+            static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err,
+                            have || pre, pa, pb, pre, pent);
+            have = false;
+        }
+    }
+    l_out = l; s_out = s; sf_out = sf;
+    if (l > 0 && !err && !drafted) {
+        if (m > 0) {                                    // the state moved: read its record, keep a copy
+            ra = __ldg(A.S.rec + 2 * (size_t)s);
+            rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
+        }
+        if (DRAFT) {
+            const int64_t e = (int64_t)ra.z;            // min_endpos
+            int64_t room = A.S.n_tokens - e;
+            my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
+            gather_draft<1>(A.S.corpus, e, my_dl, L, lane, d);
+            my_dl = cut_at_stop(d, my_dl, lane, A.W.stop_token);
+        }
+    }
+    if (m > 0 && lane == 0 && !err) {
+        cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf; cb[CB_NTOK_S] = ntok0 + (uint32_t)m;
+        if (l > 0) { reinterpret_cast<uint4*>(cb + CB_REC1)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC1)[1] = rb; }
+    }
+}
+
+// The dynamic side of one slot's step, run by one warp: Expand (fused with the dynamic matcher's Transfer)
+// for each of the slot's m tokens, then the slot's control words.  cw / cw2 are the slot's 64 control
+// words as read at the start of the step (lane i holds words i and 32 + i); on entry (ra, rb) is the copy
+// of the match state's record kept in the control block.  On exit (s2, l2) is the match state, ntok the
+// text length, and, if l2 > 0 and no error, (ra, rb) the record of s2 (also stored in the control block).
+__device__ __forceinline__ void dynamic_chain(const StepArgs& A, int b, int lane, uint32_t* cb, uint32_t cw, uint32_t cw2,
+                                              int32_t tok_first, const int32_t* toks, int m, uint32_t ntok0,
+                                              uint4& ra, uint4& rb, uint32_t (*sh_run)[12],
+                                              uint32_t& s2_out, uint32_t& l2_out, uint32_t& ntok_out, int& err) {
+    Dyn D;
+    D.pool = A.W.pool;
+    D.root = A.W.root_tab + (size_t)b * A.W.root_cap;
+    D.text = A.W.text + (size_t)b * A.W.text_stride;
+    D.pstate = A.W.pstate + (size_t)b * A.W.text_stride;
+    D.pool_hdr = A.W.pool_hdr; D.free_stack = A.W.free_stack; D.slab_owner = A.W.slab_owner;
+    D.cb = cb;
+    {   // slab table entry i is control word 16 + i
+        uint32_t lo = __shfl_sync(FULL, cw, (lane + 16) & 31), hi = __shfl_sync(FULL, cw2, (lane + 16) & 31);
+        D.tab = lane < 16 ? lo : hi;
+    }
+    D.n_rec_slabs = __shfl_sync(FULL, cw, CB_NRECSLABS);
+    D.n_states = __shfl_sync(FULL, cw, CB_NSTATES);
+    D.blk_cur = __shfl_sync(FULL, cw, CB_BLK_CUR);
+    D.blk_end = __shfl_sync(FULL, cw, CB_BLK_END);
+    D.root_deg = __shfl_sync(FULL, cw, CB_ROOTDEG);
+    D.root_bmask = (uint32_t)(A.W.root_cap / SAM_ROOT_BUCKET) - 1;
+    D.slab_shift = A.W.slab_shift; D.rps_shift = A.W.slab_shift - 5;
+    D.seq = b; D.lane = lane; D.err = 0;
+    D.pr_state = 0; D.pr_tgt = 0; D.pr_slot = 0; D.pr_bucket = SAM_NONE; D.cur = 0;
+    uint32_t last = __shfl_sync(FULL, cw, CB_LAST), ntok = ntok0;
+    uint32_t s2 = __shfl_sync(FULL, cw, CB_S2), l2 = __shfl_sync(FULL, cw, CB_L2);
+    if (D.n_states == 0) D.n_states = 1;            // the root exists implicitly (no record is read for it)
+
+    bool have = s2 != 0;
+    for (int base = 0; base < m && !D.err; base += 32) {
+        const int i = base + lane;
+        uint32_t tk = 0;
+        if (i < m) tk = (uint32_t)(base == 0 ? tok_first : toks[i]);
+        root_precompute(D, tk, i < m);              // most walks end in the root table
+        const unsigned bucket_peers = __match_any_sync(FULL, D.pr_bucket);
+        const int cnt = min(32, m - base);
+        int j = 0;
+        while (j < cnt && !D.err) {
+            if (s2 == 0) {
+                const int r = dyn_fresh_run(D, tk, j, cnt, bucket_peers, last, ntok);
+                if (r > 0) { j += r; have = false; continue; }
+                if (D.err) break;
+            }
+            Pre pre;
+            pre.valid = false;
+            if (s2 != 0 && have) {
+                const int r = dyn_repeat_run(D, tk, j, cnt, last, ntok, s2, l2, ra, rb, pre, sh_run);
+                if (r > 0) { j += r; continue; }
+                if (D.err) break;
+            }
+            D.cur = j;
+            dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2, have, ra, rb, pre);
+            j++;
+        }
+    }
+    err = D.err;
+    if (m > 0 && !err) {
+        // the newest state's record, without a transition yet
+        uint4* rl = rec_ptr(D, last);
+        if (lane == 0) {
+            rl[0] = make_uint4(ntok, s2, ntok, 0);
+            rl[1] = make_uint4(0, 0, 0, 0);
+            cb[CB_NTOK] = ntok; cb[CB_NSTATES] = D.n_states; cb[CB_LAST] = last;
+            cb[CB_S2] = s2; cb[CB_L2] = l2; cb[CB_BLK_CUR] = D.blk_cur; cb[CB_BLK_END] = D.blk_end;
+            cb[CB_NRECSLABS] = D.n_rec_slabs; cb[CB_ROOTDEG] = D.root_deg;
+        }
+        __syncwarp();
+    }
+    if (l2 > 0 && !err && m > 0) {                      // the state moved: get its record, keep a copy
+        if (!have) { const uint4* rs = rec_ptr(D, s2); ra = rs[0]; rb = rs[1]; }
+        if (lane == 0) { reinterpret_cast<uint4*>(cb + CB_REC2)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC2)[1] = rb; }
+    }
+    s2_out = s2; l2_out = l2; ntok_out = ntok;
+}
+
 // Called by one thread of a block after the block's outputs are written (and made known to that
 // thread by a block barrier where another warp wrote some of them).
 // A block orders its output stores (to mapped host memory) before its count with a device-scope fence;
@@ -813,184 +1017,20 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     if (warp == 0) {
         // ---------------- static automaton: Transfer per token ----------------
         if (A.has_static) {
-            uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
-            int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
-            bool have = s != 0;
-            // The match state is the state Build-SAM created for a whole corpus prefix (len == min_endpos:
-            // not a clone), the prefix ending at e.  Its transition on the next corpus token was created
-            // solid (len + 1) and a solid transition is never redirected, so it still leads to the state of
-            // the prefix one longer, with match length l + 1.  The state may occur more than once and have
-            // other transitions too ("ab" in "ababc"): nothing is assumed about those.  The step's tokens
-            // are compared with the corpus after e; as long as they agree the state is taken from the
-            // position -> state array, and the first token that differs goes through the ordinary Transfer
-            // below.  All in one round trip, in which the draft after e + m is requested as well in case
-            // every token agrees.
-            int j0 = 0;                      // tokens already taken
-            bool drafted = false;
-            if (have && m >= 1 && m <= 32 && ra.x == ra.z) {
-                const int64_t e = (int64_t)ra.z;
-                int32_t cx = -2; uint32_t px = 0;
-                if (lane < m && e + lane < A.S.n_tokens) { cx = __ldg(A.S.corpus + e + lane); px = __ldg(A.S.pstate + e + lane); }
-                const int64_t e2 = e + m;
-                const int64_t room = A.S.n_tokens - e2;
-                const int dl2 = (int)(room < L ? (room < 0 ? 0 : room) : L);
-                gather_draft<true>(A.S.corpus, e2, dl2, L, lane, d);
-                const unsigned agree = __ballot_sync(FULL, lane < m && cx == tok_first);
-                j0 = (~agree) ? __ffs(~agree) - 1 : 32;
-                if (j0 > 0) {
-                    const uint32_t ref = __shfl_sync(FULL, px, j0 - 1);
-                    s = ref & SAM_IDMASK; sf = ref >> 31; l += j0; have = false;
-                    if (j0 == m) {                                  // the whole step: the draft is in already
-                        ra = __ldg(A.S.rec + 2 * (size_t)s);        // its record, for the next step
-                        rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
-                        my_dl = cut_at_stop(d, dl2, lane, A.W.stop_token);
-                        drafted = true;
-                    }
-                }
-            }
-            for (int base = 0; base < m && !err && j0 < m; base += 32) {
-                const int i = base + lane;
-                uint32_t tk = 0, re = SAM_NONE;
-                if (i < m) { tk = (uint32_t)(base == 0 ? tok_first : toks[i]); re = __ldg(A.S.root_row + tk); }
-                const int cnt = min(32, m - base);
-                // Most tokens end a short match: the lookup misses, the link leads to the root, and the
-                // root row gives the next state u = root_row[t].  The token after that is then looked up
-                // in u — a lookup whose address is known now.  Lookups k = 0..7 (state root_row[t_k],
-                // token t_{k+1}) are read ahead here, eight lanes each: the state's record in lanes 0-1
-                // of the group, its hash bucket in all eight.  They are used if the matcher really is
-                // in that state when the token comes.
-                uint4 sp_rec[2], sp_ent[2];
-#pragma unroll
-                for (int r = 0; r < 2; r++) {
-                    const int k = 4 * r + (lane >> 3), e = lane & 7;
-                    const uint32_t uref = __shfl_sync(FULL, re, k);
-                    const uint32_t tnext = __shfl_sync(FULL, tk, k + 1);
-                    sp_rec[r] = make_uint4(0, 0, 0, 0);
-                    sp_ent[r] = make_uint4(SAM_NONE, 0, 0, 0);
-                    if (k + 1 < cnt && uref != SAM_NONE) {
-                        const uint32_t u = uref & SAM_IDMASK;
-                        if (e < 2) sp_rec[r] = __ldg(A.S.rec + 2 * (size_t)u + e);
-                        if (uref >> 31)
-                            sp_ent[r] = __ldg(A.S.hash + (size_t)(sam_hash2(u, tnext) & A.S.hash_mask) * SAM_HASH_BUCKET + e);
-                    }
-                }
-                for (int j = j0; j < cnt && !err; j++) {
-                    bool pre = false;
-                    uint4 pa = ra, pb = rb, pent = make_uint4(SAM_NONE, 0, 0, 0);
-                    if (j >= 1 && j <= 8 && s != 0) {
-                        const uint32_t prev = __shfl_sync(FULL, re, j - 1);
-                        if (prev != SAM_NONE && (prev & SAM_IDMASK) == s) {        // the state read ahead
-                            const int k = j - 1, g8 = 8 * (k & 3);
-                            const uint4 xr = (k >> 2) ? sp_rec[1] : sp_rec[0];
-                            const uint4 xe = (k >> 2) ? sp_ent[1] : sp_ent[0];
-                            pa.x = __shfl_sync(FULL, xr.x, g8); pa.y = __shfl_sync(FULL, xr.y, g8);
-                            pa.z = __shfl_sync(FULL, xr.z, g8); pa.w = __shfl_sync(FULL, xr.w, g8);
-                            pb.x = __shfl_sync(FULL, xr.x, g8 + 1); pb.y = __shfl_sync(FULL, xr.y, g8 + 1);
-                            pb.z = __shfl_sync(FULL, xr.z, g8 + 1); pb.w = __shfl_sync(FULL, xr.w, g8 + 1);
-                            const int src = g8 + (lane & 7);
-                            pent.x = __shfl_sync(FULL, xe.x, src); pent.y = __shfl_sync(FULL, xe.y, src);
-                            pent.z = __shfl_sync(FULL, xe.z, src); pent.w = __shfl_sync(FULL, xe.w, src);
-                            pre = true;
-                        }
-                    }
-                    static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err,
-                                    have || pre, pa, pb, pre, pent);
-                    have = false;
-                }
-            }
+            uint32_t s, sf; int32_t l;
+            static_chain<true>(A, lane, cb, cw, tok_first, toks, m, ntok0, ra, rb, s, sf, l, err, d, my_dl);
             my_l = l; my_s = (int32_t)s;
-            if (l > 0 && !err && !drafted) {
-                if (m > 0) {                                    // the state moved: read its record, keep a copy
-                    ra = __ldg(A.S.rec + 2 * (size_t)s);
-                    rb = __ldg(A.S.rec + 2 * (size_t)s + 1);
-                }
-                const int64_t e = (int64_t)ra.z;                // min_endpos
-                int64_t room = A.S.n_tokens - e;
-                my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
-                gather_draft<true>(A.S.corpus, e, my_dl, L, lane, d);
-                my_dl = cut_at_stop(d, my_dl, lane, A.W.stop_token);
-            }
-            if (m > 0 && lane == 0 && !err) {
-                cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf;
-                if (l > 0) { reinterpret_cast<uint4*>(cb + CB_REC1)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC1)[1] = rb; }
-            }
         }
     } else {
         // ---------------- dynamic automaton: Expand per token ----------------
-        Dyn D;
-        D.pool = A.W.pool;
-        D.root = A.W.root_tab + (size_t)b * A.W.root_cap;
-        D.text = A.W.text + (size_t)b * A.W.text_stride;
-        D.pstate = A.W.pstate + (size_t)b * A.W.text_stride;
-        D.pool_hdr = A.W.pool_hdr; D.free_stack = A.W.free_stack; D.slab_owner = A.W.slab_owner;
-        D.cb = cb;
-        {   // slab table entry i is control word 16 + i
-            uint32_t lo = __shfl_sync(FULL, cw, (lane + 16) & 31), hi = __shfl_sync(FULL, cw2, (lane + 16) & 31);
-            D.tab = lane < 16 ? lo : hi;
-        }
-        D.n_rec_slabs = __shfl_sync(FULL, cw, CB_NRECSLABS);
-        D.n_states = __shfl_sync(FULL, cw, CB_NSTATES);
-        D.blk_cur = __shfl_sync(FULL, cw, CB_BLK_CUR);
-        D.blk_end = __shfl_sync(FULL, cw, CB_BLK_END);
-        D.root_deg = __shfl_sync(FULL, cw, CB_ROOTDEG);
-        D.root_bmask = (uint32_t)(A.W.root_cap / SAM_ROOT_BUCKET) - 1;
-        D.slab_shift = A.W.slab_shift; D.rps_shift = A.W.slab_shift - 5;
-        D.seq = b; D.lane = lane; D.err = 0;
-        D.pr_state = 0; D.pr_tgt = 0; D.pr_slot = 0; D.pr_bucket = SAM_NONE; D.cur = 0;
-        uint32_t last = __shfl_sync(FULL, cw, CB_LAST), ntok = ntok0;
-        uint32_t s2 = __shfl_sync(FULL, cw, CB_S2), l2 = __shfl_sync(FULL, cw, CB_L2);
-        if (D.n_states == 0) D.n_states = 1;            // the root exists implicitly (no record is read for it)
-
-        bool have = s2 != 0;
-        for (int base = 0; base < m && !D.err; base += 32) {
-            const int i = base + lane;
-            uint32_t tk = 0;
-            if (i < m) tk = (uint32_t)(base == 0 ? tok_first : toks[i]);
-            root_precompute(D, tk, i < m);              // most walks end in the root table
-            const unsigned bucket_peers = __match_any_sync(FULL, D.pr_bucket);
-            const int cnt = min(32, m - base);
-            int j = 0;
-            while (j < cnt && !D.err) {
-                if (s2 == 0) {
-                    const int r = dyn_fresh_run(D, tk, j, cnt, bucket_peers, last, ntok);
-                    if (r > 0) { j += r; have = false; continue; }
-                    if (D.err) break;
-                }
-                Pre pre;
-                pre.valid = false;
-                if (s2 != 0 && have) {
-                    const int r = dyn_repeat_run(D, tk, j, cnt, last, ntok, s2, l2, ra, rb, pre, sh_run);
-                    if (r > 0) { j += r; continue; }
-                    if (D.err) break;
-                }
-                D.cur = j;
-                dyn_extend(D, __shfl_sync(FULL, tk, j), last, ntok, s2, l2, have, ra, rb, pre);
-                j++;
-            }
-        }
-        err = D.err;
+        uint32_t s2, l2, ntok;
+        dynamic_chain(A, b, lane, cb, cw, cw2, tok_first, toks, m, ntok0, ra, rb, sh_run, s2, l2, ntok, err);
         my_l = (int32_t)l2; my_s = (int32_t)s2;
-        if (m > 0 && !err) {
-            // the newest state's record, without a transition yet
-            uint4* rl = rec_ptr(D, last);
-            if (lane == 0) {
-                rl[0] = make_uint4(ntok, s2, ntok, 0);
-                rl[1] = make_uint4(0, 0, 0, 0);
-                cb[CB_NTOK] = ntok; cb[CB_NSTATES] = D.n_states; cb[CB_LAST] = last;
-                cb[CB_S2] = s2; cb[CB_L2] = l2; cb[CB_BLK_CUR] = D.blk_cur; cb[CB_BLK_END] = D.blk_end;
-                cb[CB_NRECSLABS] = D.n_rec_slabs; cb[CB_ROOTDEG] = D.root_deg;
-            }
-            __syncwarp();
-        }
         if (l2 > 0 && !err) {
-            if (m > 0) {                                        // the state moved: get its record, keep a copy
-                if (!have) { const uint4* rs = rec_ptr(D, s2); ra = rs[0]; rb = rs[1]; }
-                if (lane == 0) { reinterpret_cast<uint4*>(cb + CB_REC2)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC2)[1] = rb; }
-            }
             const int64_t e = (int64_t)ra.z;                    // min_endpos
             int64_t room = (int64_t)ntok - e;
             my_dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
-            gather_draft<false>(D.text, e, my_dl, L, lane, d);
+            gather_draft<0>(A.W.text + (size_t)b * A.W.text_stride, e, my_dl, L, lane, d);
             my_dl = cut_at_stop(d, my_dl, lane, A.W.stop_token);
         }
     }
@@ -1029,6 +1069,383 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
     }
 }
 
+// ------------------------------------------------------------------ the split step (large batches)
+// With more slots than the GPU holds blocks of the kernel above, throughput is set by how many chains are
+// resident, and a block of two warps holds two warps' worth of registers for as long as its slower chain
+// runs.  The split step gives the two sides of a slot to different blocks (of one warp) of one grid:
+//   - the dynamic side keeps its warp per slot (dynamic_chain);
+//   - the static side of a slot with few tokens needs no cooperation between lanes (a state is one 32-byte
+//     record, a hash bucket eight 16-byte entries), so one LANE carries it: a warp advances 32 slots, each
+//     round of reads serving 32 chains (static_lanes);
+//   - the static side of a slot with many tokens is what a step waits for, so it keeps a warp of its own
+//     and everything that shortens the chain (static_chain: read-ahead lookups, prefix states).
+// The slots come sorted by token count (order_slots_kernel), which also says how many of them have "many".
+// Neither side waits for the other.  Each writes its result to the slot's control block and then counts
+// itself in CB_ARRIVE; the side that finds the other already counted (an odd count) reads both results,
+// chooses the source, reads the draft and writes the slot's outputs.  Stores are ordered before the
+// count by a device-scope fence, and what the other side wrote is read with loads that bypass the L1.
+// A slot that fails its validation, or whose dynamic side runs into an error, is reported by the dynamic
+// side alone before it counts itself; the static side validates on its own (it keeps the text length in
+// CB_NTOK_S because CB_NTOK may change under it) and never commits a state for a step that is refused.
+
+__device__ __forceinline__ void write_failed_slot(const StepArgs& A, int b, int lane, int status) {
+    for (int j = lane; j < A.L; j += 32) A.draft_tokens[(size_t)b * A.L + j] = -1;
+    if (lane == 0) {
+        A.draft_len[b] = 0; A.match_len[2 * b] = 0; A.match_len[2 * b + 1] = 0; A.source[b] = 0;
+        if (A.state) { A.state[2 * b] = 0; A.state[2 * b + 1] = 0; }
+        A.status[b] = status;
+    }
+}
+
+// Count this warp's side of slot `cb` as finished; true if the other side had finished before.
+__device__ __forceinline__ bool arrive_warp(uint32_t* cb, int lane) {
+    __threadfence();
+    __syncwarp();
+    unsigned old = 0;
+    if (lane == 0) { old = atomicAdd(cb + CB_ARRIVE, 1u); __threadfence(); }
+    return (__shfl_sync(FULL, old, 0) & 1u) != 0;
+}
+
+// Both sides of slot b are done: choose the source (Section 3.2), read the draft, write the outputs.
+// Run by a whole warp.
+__device__ __forceinline__ void split_epilogue(const StepArgs& A, int b, int lane) {
+    uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const uint32_t cw = __ldcg(cb + lane), cw2 = __ldcg(cb + 32 + lane);
+    if (__shfl_sync(FULL, cw, CB_STATUS) != 0) return;                  // reported by the dynamic side
+    const int err_s = (int)__shfl_sync(FULL, cw, CB_ERR_S);
+    if (err_s) {
+        write_failed_slot(A, b, lane, err_s);
+        if (lane == 0) cb[CB_STATUS] = (uint32_t)err_s;
+        return;
+    }
+    const int l1 = (int)__shfl_sync(FULL, cw, CB_L1), l2 = (int)__shfl_sync(FULL, cw, CB_L2);
+    const int s1 = (int)__shfl_sync(FULL, cw, CB_S1), s2 = (int)__shfl_sync(FULL, cw, CB_S2);
+    const int64_t ntok = (int64_t)__shfl_sync(FULL, cw, CB_NTOK);
+    const int64_t e1 = (int64_t)__shfl_sync(FULL, cw2, CB_REC1 + 2 - 32), e2 = (int64_t)__shfl_sync(FULL, cw2, CB_REC2 + 2 - 32);
+    const int L = A.L;
+    const bool use_static = l1 > l2 + A.W.l_bias;                       // Section 3.2
+    const int lsel = use_static ? l1 : l2;
+    const int need = A.W.min_match > 1 ? A.W.min_match : 1;
+    const int src = lsel < need ? SAM_SRC_NONE : (use_static ? SAM_SRC_STATIC : SAM_SRC_DYNAMIC);
+    int32_t d[MAX_DRAFT_REGS] = {-1, -1, -1, -1};
+    int dl = 0;
+    if (src == SAM_SRC_STATIC) {
+        const int64_t room = A.S.n_tokens - e1;
+        dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
+        gather_draft<1>(A.S.corpus, e1, dl, L, lane, d);
+        dl = cut_at_stop(d, dl, lane, A.W.stop_token);
+    } else if (src == SAM_SRC_DYNAMIC) {
+        const int64_t room = ntok - e2;
+        dl = (int)(room < L ? (room < 0 ? 0 : room) : L);
+        gather_draft<2>(A.W.text + (size_t)b * A.W.text_stride, e2, dl, L, lane, d);
+        dl = cut_at_stop(d, dl, lane, A.W.stop_token);
+    }
+#pragma unroll
+    for (int r = 0; r < MAX_DRAFT_REGS; r++) {
+        const int j = r * 32 + lane;
+        if (j < L) A.draft_tokens[(size_t)b * L + j] = d[r];
+    }
+    if (lane == 0) {
+        A.draft_len[b] = dl; A.match_len[2 * b] = l1; A.match_len[2 * b + 1] = l2; A.source[b] = src;
+        if (A.state) { A.state[2 * b] = s1; A.state[2 * b + 1] = s2; }
+        A.status[b] = 0;
+    }
+}
+
+// The same for the slots of the lanes of a static_lanes warp that found their dynamic side done (`second`).
+// Each such lane knows its own side's result (l1, s1, e1, err_s) and reads the other's from its control block;
+// the drafts are then read by the whole warp, row after row — lane k reads token k of every pending row, all
+// rows' reads issued together — and written the same way.
+__device__ __forceinline__ void split_epilogue_lanes(const StepArgs& A, bool second, int b, int lane,
+                                                     int l1, int s1, int64_t e1, int err_s) {
+    const unsigned pending0 = __ballot_sync(FULL, second);
+    if (!pending0) return;
+    uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const int L = A.L;
+    int l2 = 0, s2 = 0, src = SAM_SRC_NONE, dl = 0, status = 0;
+    int64_t e = 0;
+    const int32_t* text = A.S.corpus;
+    bool mine = second;
+    if (second) {
+        const uint32_t st = __ldcg(cb + CB_STATUS);
+        l2 = (int)__ldcg(cb + CB_L2); s2 = (int)__ldcg(cb + CB_S2);
+        const int64_t ntok = (int64_t)__ldcg(cb + CB_NTOK), e2 = (int64_t)__ldcg(cb + CB_REC2 + 2);
+        if (st != 0) mine = false;                                       // reported by the dynamic side
+        else if (err_s) { status = err_s; l1 = l2 = 0; s1 = s2 = 0; cb[CB_STATUS] = (uint32_t)err_s; }
+        else {
+            const bool use_static = l1 > l2 + A.W.l_bias;               // Section 3.2
+            const int lsel = use_static ? l1 : l2;
+            const int need = A.W.min_match > 1 ? A.W.min_match : 1;
+            src = lsel < need ? SAM_SRC_NONE : (use_static ? SAM_SRC_STATIC : SAM_SRC_DYNAMIC);
+            if (!use_static) text = A.W.text + (size_t)b * A.W.text_stride;
+            e = use_static ? e1 : e2;
+            const int64_t room = (use_static ? A.S.n_tokens : ntok) - e;
+            dl = src == SAM_SRC_NONE ? 0 : (int)(room < L ? (room < 0 ? 0 : room) : L);
+        }
+    }
+    const unsigned pending = __ballot_sync(FULL, mine);
+    const int32_t* src_ptr = text + e;
+    int32_t* row = A.draft_tokens + (size_t)b * L;
+    const int32_t stop = A.W.stop_token;
+    int cut = dl;                                                        // this lane's row ends here
+    for (int base = 0; base < L; base += 32) {
+        int32_t v[32];
+#pragma unroll
+        for (int i = 0; i < 32; i++) {                                   // row i, token base + lane
+            const int32_t* p_i = reinterpret_cast<const int32_t*>(__shfl_sync(FULL, (unsigned long long)src_ptr, i));
+            const int dl_i = __shfl_sync(FULL, dl, i);
+            v[i] = -1;
+            if (base + lane < dl_i) v[i] = __ldcg(p_i + base + lane);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; i++) {
+            int cut_i = __shfl_sync(FULL, cut, i);
+            const unsigned hit = __ballot_sync(FULL, stop >= 0 && v[i] == stop && base + lane < cut_i);
+            if (hit) cut_i = base + __ffs(hit) - 1;                      // a draft ends before the first stop token
+            if (lane == i) cut = cut_i;
+            int32_t* row_i = reinterpret_cast<int32_t*>(__shfl_sync(FULL, (unsigned long long)row, i));
+            if (((pending >> i) & 1u) && base + lane < L) row_i[base + lane] = base + lane < cut_i ? v[i] : -1;
+        }
+    }
+    if (mine) {
+        A.draft_len[b] = cut; A.match_len[2 * b] = l1; A.match_len[2 * b + 1] = l2; A.source[b] = src;
+        if (A.state) { A.state[2 * b] = s1; A.state[2 * b + 1] = s2; }
+        A.status[b] = status;
+    }
+}
+
+// The static side of 32 slots, one per lane: Transfer (Algorithm 1) for each of the slot's tokens.
+// Every pass of the loop is one round of reads for all lanes that still have tokens: the record of the
+// lane's state, the home bucket of (state, token) when the state has hashed transitions, the root-row
+// entry of the token (used when the walk reaches the root in this pass) and the slot's next token.
+__device__ __forceinline__ void static_lanes(const StepArgs& A, int w, int lane) {
+    const SamStaticView& S = A.S;
+    const int idx = A.W.batch - 1 - (w * 32 + lane);      // from the end of the sorted order: the fewest tokens first
+    const int ob = A.order[idx > 0 ? idx : 0];            // (read together with the count below)
+    const int first = min(*A.split_count, A.n_warp_blocks);   // the slots before this one have a warp of their own
+    const bool live = idx >= first;
+    if (!__any_sync(FULL, live)) return;
+    const int b = live ? ob : 0;
+    uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
+    uint32_t status = 0, s = 0, sf = 0, ntok_s = 0;
+    int32_t l = 0, t = 0;
+    int m = 0;
+    uint4 ra = make_uint4(0, 0, 0, 0), rb = ra;
+    if (live) {
+        status = cb[CB_STATUS]; s = cb[CB_S1]; l = (int32_t)cb[CB_L1]; sf = cb[CB_S1FLAG]; ntok_s = cb[CB_NTOK_S];
+        ra = *reinterpret_cast<const uint4*>(cb + CB_REC1); rb = *reinterpret_cast<const uint4*>(cb + CB_REC1 + 4);
+        m = A.counts[b];
+        t = toks[0];
+    }
+    // the same checks, in the same order, as the dynamic side makes (bad count, capacity, then the tokens
+    // one by one as they come up): a refused step leaves the static state as it was
+    bool run = live && status == 0 && m >= 0 && m <= A.stride && (int64_t)ntok_s + m <= A.W.max_seq_len;
+    bool active = run && m > 0;
+    if (active && (t < 0 || t >= S.vocab)) { active = false; run = false; }
+    bool have = s != 0;                                  // (ra, rb) is the record of s
+    bool need_len = false;
+    int j = 0, err = 0;
+    int guard = l + 2 * m + 4;                           // at most l + m link moves in all (Appendix A.3)
+    while (__any_sync(FULL, active)) {
+        // One round of reads for every lane, none of them under a branch (lanes that took different branches
+        // would otherwise wait for their reads one group after the other): a lane that does not need a line
+        // reads one that every such lane shares (record 0, bucket 0, its own first token).
+        const bool at_root = s == 0;
+        const bool want_rec = active && !at_root && !have;
+        const bool want_bucket = active && !at_root && sf != 0;
+        uint32_t home = want_bucket ? sam_hash2(s, (uint32_t)t) & S.hash_mask : 0u;
+        const uint32_t re = __ldg(S.root_row + (active ? t : 0));
+        const int32_t tn = toks[(active && j + 1 < m) ? j + 1 : 0];
+        const size_t ri = want_rec ? (size_t)s : 0;
+        uint4 a = __ldg(S.rec + 2 * ri), bb = __ldg(S.rec + 2 * ri + 1);
+        uint4 ent[SAM_HASH_BUCKET];
+#pragma unroll
+        for (int e = 0; e < SAM_HASH_BUCKET; e++) ent[e] = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + e);
+        if (have) { a = ra; bb = rb; }
+        if (active) {
+            have = false;
+            bool advance = false;
+            if (at_root) {                                // at the root the match length is 0
+                if (re != SAM_NONE) { s = re & SAM_IDMASK; sf = re >> 31; l = 1; } else l = 0;
+                advance = true;
+            } else {
+                if (need_len) { l = (int32_t)a.x; need_len = false; }
+                uint32_t tgt = SAM_NONE;
+                if (a.w >= 1 && bb.x == (uint32_t)t) tgt = bb.y;
+                else if (a.w >= 2 && bb.z == (uint32_t)t) tgt = bb.w;
+                else if (a.w > 2) {
+                    if (!sf) {                            // (every reference to a state with hashed transitions carries the flag)
+                        home = sam_hash2(s, (uint32_t)t) & S.hash_mask;
+#pragma unroll
+                        for (int e = 0; e < SAM_HASH_BUCKET; e++) ent[e] = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + e);
+                    }
+                    for (int probe = 1;; probe++) {
+                        bool empty = false;
+#pragma unroll
+                        for (int e = 0; e < SAM_HASH_BUCKET; e++) {
+                            if (ent[e].x == s && ent[e].y == (uint32_t)t) tgt = ent[e].z;
+                            empty |= ent[e].x == SAM_NONE;
+                        }
+                        if (tgt != SAM_NONE || empty || probe >= S.hash_max_probe) break;
+                        home = (home + 1) & S.hash_mask;
+#pragma unroll
+                        for (int e = 0; e < SAM_HASH_BUCKET; e++) ent[e] = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + e);
+                    }
+                }
+                if (tgt != SAM_NONE) { s = tgt & SAM_IDMASK; sf = tgt >> 31; l += 1; advance = true; }
+                else {                                    // s <- link(s), l <- len(link(s))
+                    s = a.y & SAM_IDMASK; sf = a.y >> 31;
+                    if (s == 0) {                         // the root either has the token or not: known already
+                        if (re != SAM_NONE) { s = re & SAM_IDMASK; sf = re >> 31; l = 1; } else l = 0;
+                        advance = true;
+                    } else need_len = true;
+                    if (--guard < 0) { err = SAM_SEQ_WALK_LIMIT; active = false; }
+                }
+            }
+            if (advance && active) {
+                if (++j < m) {
+                    t = tn;
+                    if (t < 0 || t >= S.vocab) { active = false; run = false; }
+                } else active = false;
+            }
+        }
+    }
+    int64_t e1 = (int64_t)ra.z;
+    if (run && m > 0 && !err) {
+        if (l > 0) {                                      // the state moved: read its record, keep a copy
+            ra = __ldg(S.rec + 2 * (size_t)s); rb = __ldg(S.rec + 2 * (size_t)s + 1);
+            *reinterpret_cast<uint4*>(cb + CB_REC1) = ra; *reinterpret_cast<uint4*>(cb + CB_REC1 + 4) = rb;
+            e1 = (int64_t)ra.z;
+        }
+        cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf; cb[CB_NTOK_S] = ntok_s + (uint32_t)m;
+    }
+    if (live && err) cb[CB_ERR_S] = (uint32_t)err;
+    bool second = false;
+    if (live) {
+        __threadfence();
+        second = (atomicAdd(cb + CB_ARRIVE, 1u) & 1u) != 0;
+        __threadfence();
+    }
+    split_epilogue_lanes(A, second, b, lane, l, (int32_t)s, e1, err);
+}
+
+// The dynamic side of one slot (one warp), including everything that reports a slot as failed.
+__device__ __forceinline__ void dynamic_slot(const StepArgs& A, int b, int lane, uint32_t (*sh_run)[12]) {
+    uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
+    const uint32_t cw = cb[lane];
+    const uint32_t cw2 = cb[32 + lane];
+    int32_t tok_first = 0;
+    if (lane < A.stride) tok_first = toks[lane];
+    const int m = A.counts[b];
+    int status = (int)__shfl_sync(FULL, cw, CB_STATUS);
+    const uint32_t ntok0 = __shfl_sync(FULL, cw, CB_NTOK);
+    bool fresh_fail = false;
+    if (status == 0) {                                   // validate the whole step before any state changes
+        if (m < 0 || m > A.stride) status = SAM_SEQ_BAD_COUNT;
+        else if ((int64_t)ntok0 + m > A.W.max_seq_len) status = SAM_SEQ_CAPACITY;
+        else {
+            bool bad = false;
+            for (int base = 0; base < m; base += 32) {
+                const int i = base + lane;
+                if (i < m) { const int tt = base == 0 ? tok_first : toks[i]; bad |= (tt < 0 || tt >= A.S.vocab); }
+            }
+            if (__any_sync(FULL, bad)) status = SAM_SEQ_BAD_TOKEN;
+        }
+        fresh_fail = status != 0;
+    }
+    int err = 0;
+    if (status == 0) {
+        const int rbase = CB_REC2 - 32;
+        uint4 ra, rb;
+        ra.x = __shfl_sync(FULL, cw2, rbase + 0); ra.y = __shfl_sync(FULL, cw2, rbase + 1);
+        ra.z = __shfl_sync(FULL, cw2, rbase + 2); ra.w = __shfl_sync(FULL, cw2, rbase + 3);
+        rb.x = __shfl_sync(FULL, cw2, rbase + 4); rb.y = __shfl_sync(FULL, cw2, rbase + 5);
+        rb.z = __shfl_sync(FULL, cw2, rbase + 6); rb.w = __shfl_sync(FULL, cw2, rbase + 7);
+        uint32_t s2, l2, ntok;
+        dynamic_chain(A, b, lane, cb, cw, cw2, tok_first, toks, m, ntok0, ra, rb, sh_run, s2, l2, ntok, err);
+        if (err) { status = err; fresh_fail = true; }
+    }
+    if (status != 0) {
+        if (fresh_fail && lane == 0) cb[CB_STATUS] = (uint32_t)status;
+        write_failed_slot(A, b, lane, status);
+        arrive_warp(cb, lane);
+        return;
+    }
+    if (arrive_warp(cb, lane)) split_epilogue(A, b, lane);
+}
+
+// The static side of one slot with a warp of its own.
+__device__ __forceinline__ void static_slot(const StepArgs& A, int b, int lane) {
+    uint32_t* cb = A.W.ctrl + (size_t)b * SAM_CTRL_WORDS;
+    const int32_t* toks = A.new_tokens + (size_t)b * A.stride;
+    const uint32_t cw = cb[lane];
+    const uint32_t cw2 = cb[32 + lane];
+    int32_t tok_first = 0;
+    if (lane < A.stride) tok_first = toks[lane];
+    const int m = A.counts[b];
+    const uint32_t ntok_s = __shfl_sync(FULL, cw, CB_NTOK_S);
+    bool run = __shfl_sync(FULL, cw, CB_STATUS) == 0 && m >= 0 && m <= A.stride && (int64_t)ntok_s + m <= A.W.max_seq_len;
+    if (run) {                                           // the dynamic side reports a refused step; this side only keeps out
+        bool bad = false;
+        for (int base = 0; base < m; base += 32) {
+            const int i = base + lane;
+            if (i < m) { const int tt = base == 0 ? tok_first : toks[i]; bad |= (tt < 0 || tt >= A.S.vocab); }
+        }
+        run = !__any_sync(FULL, bad);
+    }
+    if (run) {
+        const int rbase = CB_REC1 - 32;
+        uint4 ra, rb;
+        ra.x = __shfl_sync(FULL, cw2, rbase + 0); ra.y = __shfl_sync(FULL, cw2, rbase + 1);
+        ra.z = __shfl_sync(FULL, cw2, rbase + 2); ra.w = __shfl_sync(FULL, cw2, rbase + 3);
+        rb.x = __shfl_sync(FULL, cw2, rbase + 4); rb.y = __shfl_sync(FULL, cw2, rbase + 5);
+        rb.z = __shfl_sync(FULL, cw2, rbase + 6); rb.w = __shfl_sync(FULL, cw2, rbase + 7);
+        uint32_t s, sf; int32_t l, dl = 0;
+        int32_t d[MAX_DRAFT_REGS];
+        int err = 0;
+        static_chain<false>(A, lane, cb, cw, tok_first, toks, m, ntok_s, ra, rb, s, sf, l, err, d, dl);
+        if (err && lane == 0) cb[CB_ERR_S] = (uint32_t)err;
+    }
+    if (arrive_warp(cb, lane)) split_epilogue(A, b, lane);
+}
+
+__global__ void __launch_bounds__(32) sam_step_split_kernel(const __grid_constant__ StepArgs A) {
+    {   // while the previous kernel of the stream finishes: a dynamic-side block touches (prefetch, no data is
+        // used) the lines it reads first
+        const int pi = (int)blockIdx.x - A.n_warp_blocks - A.n_lane_blocks, pl = (int)threadIdx.x;
+        if (pi >= 0 && pl < 4) {
+            const char* p0 = reinterpret_cast<const char*>(A.W.ctrl + (size_t)pi * SAM_CTRL_WORDS);
+            const char* p1 = reinterpret_cast<const char*>(A.new_tokens + (size_t)pi * A.stride);
+            const char* p2 = reinterpret_cast<const char*>(A.counts + pi);
+            const char* pp = pl == 0 ? p0 : pl == 1 ? p0 + 128 : pl == 2 ? p1 : p2;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(pp));
+        }
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+    __shared__ __align__(16) uint32_t sh_run[32][12];   // per-token staging of a repeat run (dynamic side)
+    const int lane = threadIdx.x;
+    int i = (int)blockIdx.x;
+    if (i < A.n_warp_blocks + A.n_lane_blocks) {
+        // slots whose static side gets a warp: the first n_big of the sorted order (read together with order[])
+        if (i < A.n_warp_blocks) {
+            const int b = A.order[i];
+            if (i < min(*A.split_count, A.n_warp_blocks)) static_slot(A, b, lane);
+        } else {
+            static_lanes(A, i - A.n_warp_blocks, lane);
+        }
+    } else {
+        // the dynamic side's time hardly depends on the token count: slots in their own order, one read less
+        dynamic_slot(A, i - A.n_warp_blocks - A.n_lane_blocks, lane, sh_run);
+    }
+    if (A.done_flag) {
+        __syncwarp();
+        if (lane == 0) signal_done(A);
+    }
+}
+
 // A batch larger than the GPU holds at once runs in waves, and a step is as long as its last block: a
 // slot with many tokens that starts in the last wave ends late.  This kernel sorts the slots by their
 // token count, largest first (a counting sort in shared memory), so that block i of the step kernel takes
@@ -1042,7 +1459,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
 // counts itself, after its own dependency wait).
 constexpr int SAM_ORDER_KEYS = 64;
 __global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts, int32_t B, int32_t* order,
-                                                           int32_t* keys) {
+                                                           int32_t* keys, int32_t big_m, int32_t* n_big) {
     asm volatile("griddepcontrol.launch_dependents;");
     __shared__ int hist[SAM_ORDER_KEYS];
     for (int k = threadIdx.x; k < SAM_ORDER_KEYS; k += blockDim.x) hist[k] = 0;
@@ -1056,7 +1473,10 @@ __global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts
     __syncthreads();
     if (threadIdx.x == 0) {                                  // hist[k] <- first position of key k, keys descending
         int at = 0;
-        for (int k = SAM_ORDER_KEYS - 1; k >= 0; k--) { const int n = hist[k]; hist[k] = at; at += n; }
+        for (int k = SAM_ORDER_KEYS - 1; k >= 0; k--) {
+            const int n = hist[k]; hist[k] = at; at += n;
+            if (k == big_m) *n_big = at;                     // slots with at least big_m tokens: the first `at` of order[]
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < B; i += blockDim.x) {
@@ -1066,8 +1486,31 @@ __global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// From how many tokens on a slot's static side gets a warp of its own in the split step.  A lane's chain costs
+// about 1.3 us per read round against 0.5 us per token for a warp's; up to a few thousand slots a step is as
+// long as its slowest slot, beyond that the number of resident warps counts for more.
+constexpr int split_big_m(int batch) { return batch >= 8192 ? 8 : 5; }
+
+// The split kernel's blocks are single warps with 1.5 KB of shared memory each: the default split between L1
+// and shared memory would hold only a dozen of them per SM.  Once per device.
+int split_kernel_setup(int device);
+
+constexpr int SAM_SPLIT_MIN_BATCH = 8192;                    // the split step is used from this many slots on
 constexpr int SAM_ORDER_MIN_BATCH = 1536;                    // more slots than a B200 holds blocks of this kernel (148 x 10)
 
+}  // namespace
+
+namespace {
+int split_kernel_setup(int device) {
+    static bool done[64];
+    if (device < 0 || device >= 64) return SAM_ERR_ARG;
+    if (!done[device]) {
+        cudaError_t e = cudaFuncSetAttribute(sam_step_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50);
+        if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
+        done[device] = true;
+    }
+    return SAM_OK;
+}
 }  // namespace
 
 int sam_step_launch_count(const sam_batch* b) { return b->view.batch >= SAM_ORDER_MIN_BATCH ? 2 : 1; }
@@ -1107,15 +1550,17 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    A.order = nullptr;
+    A.order = nullptr; A.split_count = nullptr;
     if (!v_draft && b->view.batch >= SAM_ORDER_MIN_BATCH) {
         int32_t* order = b->view.order + (size_t)(b->order_phase & 1) * b->view.batch;
-        b->order_phase ^= 1;
         cudaLaunchConfig_t oc;
         memset(&oc, 0, sizeof(oc));
         oc.gridDim = dim3(1); oc.blockDim = dim3(1024); oc.stream = stream; oc.attrs = attr; oc.numAttrs = 1;
+        int32_t* n_big = b->view.order + 3 * (size_t)b->view.batch + 8 * (b->order_phase & 1);
         cudaError_t oe = cudaLaunchKernelEx(&oc, order_slots_kernel, counts, (int32_t)b->view.batch, order,
-                                            b->view.order + 2 * (size_t)b->view.batch);
+                                            b->view.order + 2 * (size_t)b->view.batch, split_big_m(b->view.batch), n_big);
+        A.split_count = n_big;
+        b->order_phase ^= 1;
         if (oe != cudaSuccess) { sam_set_cuda_error(oe); return SAM_ERR_CUDA; }
         A.order = order;
     }
@@ -1123,8 +1568,19 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)b->view.batch); cfg.blockDim = dim3(64); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = v_draft ? cudaLaunchKernelEx(&cfg, sam_step_kernel<true>, A)
-                            : cudaLaunchKernelEx(&cfg, sam_step_kernel<false>, A);
+    A.n_warp_blocks = A.n_lane_blocks = 0;
+    cudaError_t e;
+    if (A.order && A.has_static && b->view.batch >= SAM_SPLIT_MIN_BATCH) {   // the two sides of a slot in different blocks
+        int rc = split_kernel_setup(b->device);
+        if (rc) return rc;
+        A.n_warp_blocks = (b->view.batch + 3) / 4;
+        A.n_lane_blocks = (b->view.batch + 31) / 32;
+        cfg.gridDim = dim3((unsigned)(b->view.batch + A.n_warp_blocks + A.n_lane_blocks)); cfg.blockDim = dim3(32);
+        e = cudaLaunchKernelEx(&cfg, sam_step_split_kernel, A);
+    } else {
+        e = v_draft ? cudaLaunchKernelEx(&cfg, sam_step_kernel<true>, A)
+                    : cudaLaunchKernelEx(&cfg, sam_step_kernel<false>, A);
+    }
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
     return SAM_OK;

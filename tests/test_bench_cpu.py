@@ -56,3 +56,34 @@ def test_recipes_have_the_stated_shape():
     c2 = W.make(W.scaled(W.SPECS["tiny"], corpus_len=5000, seed=7))
     assert np.array_equal(a.corpus, b.corpus) and np.array_equal(a.seqs, b.seqs)
     assert not np.array_equal(a.corpus, c2.corpus)
+
+
+def test_multi_document_recipe_joins_documents_with_the_separator():
+    """The sixth recipe: separators stand at document ends only, documents have the stated lengths, and
+    the CPU oracle run with the separator as stop token never drafts across a document boundary."""
+    import oracle
+    spec = W.scaled(W.DOCS, corpus_len=200_000, batch=6, prompt_len=150, gen_len=250)
+    w = W.make(spec)
+    ends = np.flatnonzero(w.corpus == spec.eos)
+    assert ends[-1] == spec.corpus_len - 1
+    lens = np.diff(np.concatenate([[-1], ends]))
+    assert lens[:-1].min() >= spec.doc_lo and lens.max() <= spec.doc_hi
+    S = oracle.Sam(w.corpus)
+    L, B = spec.draft_len, spec.batch
+    ob = oracle.Batch(S, w.corpus, B, spec.vocab, spec.prompt_len + spec.gen_len, stop_token=spec.eos)
+    free = oracle.Batch(S, w.corpus, B, spec.vocab, spec.prompt_len + spec.gen_len)
+    outs = [ob.step(w.prompts, np.full(B, spec.prompt_len, dtype=np.int32), L)]
+    plain = [free.step(w.prompts, np.full(B, spec.prompt_len, dtype=np.int32), L)]
+    for s in range(w.n_steps):
+        outs.append(ob.step(w.new_tokens[s], w.counts[s], L))
+        plain.append(free.step(w.new_tokens[s], w.counts[s], L))
+    cut = 0
+    for o, q in zip(outs, plain):
+        assert not (o.draft_tokens == spec.eos).any()
+        assert np.array_equal(o.match_len, q.match_len) and np.array_equal(o.source, q.source)
+        for b in range(B):
+            d, full = o.draft_tokens[b, :o.draft_len[b]], q.draft_tokens[b, :q.draft_len[b]]
+            hit = np.flatnonzero(full == spec.eos)
+            assert np.array_equal(d, full[:hit[0]] if len(hit) else full)     # the plain slice, cut at the separator
+            cut += len(hit) > 0
+    assert cut > 0

@@ -275,6 +275,26 @@ def test_workload_recipes(P, name):
     assert info.n_states == S.n_states and info.n_transitions == S.n_transitions
 
 
+def test_multi_document_corpus_with_stop_token(P):
+    """A corpus of documents joined by an end-of-sequence token, with that token as the drafts' stop
+    token (Section 3.1): every output equals the oracle's, no draft crosses a document boundary, and
+    some drafts are in fact cut short by a separator."""
+    spec = W.scaled(W.DOCS, 600_000, 24, 500, 700)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, ob, S = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=4, stop_token=spec.eos)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, stop_token=spec.eos)
+    assert_same(got, ref, "docs")
+    assert (got["status"] == 0).all() and not (got["draft_tokens"] == spec.eos).any()
+    tb = P.binding.sam_static_tables(st.handle)
+    stat = got["source"] == 1
+    e1 = tb["min_endpos"][got["state"][..., 0]]
+    room = np.minimum(L, spec.corpus_len - e1)
+    assert (stat & (got["draft_len"] < room)).any()                 # cut by a separator, not by the corpus' end
+    assert st.info.n_states == S.n_states and st.info.n_transitions == S.n_transitions
+
+
 def test_c2_full_size_bench_configuration(P):
     """Config 2 at full size, launched exactly as the benchmark launches it (prefill step, then one
     launch per decoding step through sam_run_steps): every output of every step equals the oracle."""

@@ -43,6 +43,9 @@ def _load():
         lib.samgen_model_free.argtypes = [ctypes.c_void_p]
         lib.samgen_corpus.argtypes = [ctypes.c_void_p, i32p, ctypes.c_int64, ctypes.c_double,
                                       ctypes.c_int32, ctypes.c_int32, ctypes.c_uint64]
+        lib.samgen_join_documents.restype = ctypes.c_int64
+        lib.samgen_join_documents.argtypes = [i32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                              ctypes.c_int32, ctypes.c_uint64]
         lib.samgen_sequences.argtypes = [ctypes.c_void_p, i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                          i32p, ctypes.c_int64, ctypes.c_double, ctypes.c_double,
                                          ctypes.c_double, ctypes.c_double, ctypes.c_int32,
@@ -86,6 +89,9 @@ class Spec:
     draft_len: int
     unrelated_corpus: bool = False  # corpus drawn with another permutation: no useful static hits
     seed: int = 0
+    doc_lo: int = 0                # > 0: the corpus is documents of U[doc_lo, doc_hi] tokens joined by `eos`
+    doc_hi: int = 0
+    eos: int = -1                  # the separator's token id (also the drafts' stop token)
 
 
 # The five recipes, smallest first; seeds are 0x5A4D0000 + position.
@@ -102,6 +108,14 @@ SPECS = {
     "c5": Spec("c5", 200_000_000, 128256, 1.05, True, 0.25, 8, 256, 4096, 2048, 2048,
                0.40, 0.5, 0.40, 0.5, True, "geometric", 16, 0.3, 32, seed=0x5A4D0004),
 }
+
+# A sixth recipe, not one of the five benchmark configurations: c2's shape over a corpus that is many
+# documents joined by an end-of-sequence token (id vocab - 1), the way a retrieval corpus is put
+# together from separate texts.  Run with the stop token set to `eos`, so that no draft crosses a
+# document boundary.
+DOCS = Spec("docs", 4_000_000, 32000, 1.1, True, 0.25, 8, 128, 64, 1024, 2048,
+            0.35, 0.5, 0.35, 0.5, False, "geometric", 8, 0.4, 32, seed=0x5A4D0005,
+            doc_lo=40, doc_hi=1200, eos=31999)
 
 
 def scaled(spec: Spec, corpus_len=None, batch=None, prompt_len=None, gen_len=None, seed=None) -> Spec:
@@ -151,6 +165,8 @@ def make_corpus(spec: Spec) -> np.ndarray:
         corpus = np.empty(spec.corpus_len, dtype=np.int32)
         lib.samgen_corpus(model, _p(corpus), spec.corpus_len, spec.corpus_copy_frac,
                           spec.span_lo, spec.span_hi, seed)
+        if spec.doc_lo > 0:
+            lib.samgen_join_documents(_p(corpus), spec.corpus_len, spec.vocab, spec.eos, spec.doc_lo, spec.doc_hi, seed)
     finally:
         lib.samgen_model_free(model)
     return corpus

@@ -145,6 +145,25 @@ void samgen_corpus(void* model, int32_t* out, int64_t n, double f, int32_t lo, i
     fill_text((const model_t*)model, &g, out, 0, n, f, lo, hi, NULL, 0, 0.0, 0, -1);
 }
 
+/* Multi-document corpus: the text is cut into documents whose lengths (separator included) are
+ * U[lo, hi], and the last token of each document is replaced by the separator id `eos` — a corpus
+ * of many documents joined into one string by an end-of-sequence token.  Any `eos` the token model
+ * itself drew inside a document is replaced by (eos + 1) mod vocab, so the separator occurs at
+ * document ends only.  Returns the number of documents. */
+int64_t samgen_join_documents(int32_t* corpus, int64_t n, int32_t vocab, int32_t eos, int32_t lo, int32_t hi,
+                              uint64_t seed) {
+    rng_t g; rng_init(&g, seed, 0x646F6373ull /* "docs" */);
+    int64_t docs = 0, i = 0;
+    while (i < n) {
+        int64_t len = rng_range(&g, lo, hi);
+        int64_t end = i + len < n ? i + len : n;
+        for (int64_t k = i; k < end - 1; k++) if (corpus[k] == eos) corpus[k] = (eos + 1) % vocab;
+        corpus[end - 1] = eos;
+        i = end; docs++;
+    }
+    return docs;
+}
+
 /* Sequences: out is [batch, prompt_len + gen_len] row-major.
  * Prompt tokens use (f_prompt, p_other_prompt); generated tokens use (f_gen, p_other_gen).
  * own_prompt_only != 0 restricts own-text copies in the generated part to the prompt. */
