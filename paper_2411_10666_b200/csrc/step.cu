@@ -1097,12 +1097,31 @@ __device__ __forceinline__ void write_failed_slot(const StepArgs& A, int b, int 
     }
 }
 
+// How many sides of the slot have counted themselves, read with acquire semantics: if the count is odd the
+// other side is done and everything it wrote may be read from here on (with loads that bypass the L1).
+__device__ __forceinline__ uint32_t arrive_look(const uint32_t* cb) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(cb + CB_ARRIVE) : "memory");
+    return v;
+}
+
 // Count this warp's side of slot `cb` as finished; true if the other side had finished before.
+// A side that finds the other one done already (an acquiring look, one read) has no reader for what it wrote
+// in this kernel: it counts itself without waiting for its stores.  Otherwise its stores are ordered before
+// the count by a device-scope fence — the wait for them to be acknowledged is what that costs — and the
+// count's old value decides.
 __device__ __forceinline__ bool arrive_warp(uint32_t* cb, int lane) {
+    uint32_t seen = 0;
+    if (lane == 0) seen = arrive_look(cb);
+    seen = __shfl_sync(FULL, seen, 0);
+    if (seen & 1u) {
+        if (lane == 0) atomicAdd(cb + CB_ARRIVE, 1u);
+        return true;
+    }
     __threadfence();
     __syncwarp();
     unsigned old = 0;
-    if (lane == 0) { old = atomicAdd(cb + CB_ARRIVE, 1u); __threadfence(); }
+    if (lane == 0) { old = atomicAdd(cb + CB_ARRIVE, 1u); if (old & 1u) __threadfence(); }
     return (__shfl_sync(FULL, old, 0) & 1u) != 0;
 }
 
@@ -1323,9 +1342,12 @@ __device__ __forceinline__ void static_lanes(const StepArgs& A, int w, int lane)
     if (live && err) cb[CB_ERR_S] = (uint32_t)err;
     bool second = false;
     if (live) {
-        __threadfence();
-        second = (atomicAdd(cb + CB_ARRIVE, 1u) & 1u) != 0;
-        __threadfence();
+        if (arrive_look(cb) & 1u) { atomicAdd(cb + CB_ARRIVE, 1u); second = true; }
+        else {
+            __threadfence();
+            second = (atomicAdd(cb + CB_ARRIVE, 1u) & 1u) != 0;
+            if (second) __threadfence();
+        }
     }
     split_epilogue_lanes(A, second, b, lane, l, (int32_t)s, e1, err);
 }
@@ -1458,17 +1480,39 @@ __global__ void __launch_bounds__(32) sam_step_split_kernel(const __grid_constan
 // a count read too early only costs the intended launch order, never a result (the step kernel reads the
 // counts itself, after its own dependency wait).
 constexpr int SAM_ORDER_KEYS = 64;
-__global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts, int32_t B, int32_t* order,
-                                                           int32_t* keys, int32_t big_m, int32_t* n_big) {
+constexpr int SAM_ORDER_THREADS = 1024;
+// (SPLIT: the instance launched ahead of the split step; it is given that kernel's split between L1 and shared
+// memory, because kernels that want different ones do not share an SM.)
+template <bool SPLIT>
+__global__ void __launch_bounds__(SAM_ORDER_THREADS) order_slots_kernel(const int32_t* counts, int32_t B, int32_t* order,
+                                                                        int32_t* keys, int32_t big_m, int32_t* n_big) {
     asm volatile("griddepcontrol.launch_dependents;");
     __shared__ int hist[SAM_ORDER_KEYS];
+    const int lane = threadIdx.x & 31;
+    const unsigned lt = (1u << lane) - 1u;
     for (int k = threadIdx.x; k < SAM_ORDER_KEYS; k += blockDim.x) hist[k] = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < B; i += blockDim.x) {
-        const int m = *reinterpret_cast<const volatile int32_t*>(counts + i);
-        const int key = m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m);
-        keys[i] = key;                                       // read back by this same thread below
-        atomicAdd(&hist[key], 1);
+    // Four slots per thread and round, so that four reads are under way at a time; the lanes of a warp that
+    // hold the same key count themselves with one addition (the counts cluster on a few small values).
+    constexpr int U = 4;
+    for (int base = 0; base < B; base += U * SAM_ORDER_THREADS) {
+        int key[U];
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const int i = base + u * SAM_ORDER_THREADS + (int)threadIdx.x;
+            key[u] = -1;
+            if (i < B) {
+                const int m = *reinterpret_cast<const volatile int32_t*>(counts + i);
+                key[u] = m < 0 ? 0 : (m >= SAM_ORDER_KEYS ? SAM_ORDER_KEYS - 1 : m);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const int i = base + u * SAM_ORDER_THREADS + (int)threadIdx.x;
+            if (i < B) keys[i] = key[u];                     // read back by this same thread below
+            const unsigned peers = __match_any_sync(FULL, key[u]);
+            if (key[u] >= 0 && (peers & lt) == 0) atomicAdd(&hist[key[u]], __popc(peers));
+        }
     }
     __syncthreads();
     if (threadIdx.x == 0) {                                  // hist[k] <- first position of key k, keys descending
@@ -1479,9 +1523,23 @@ __global__ void __launch_bounds__(1024) order_slots_kernel(const int32_t* counts
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < B; i += blockDim.x) {
-        const int pos = atomicAdd(&hist[keys[i]], 1);
-        if (pos < B) order[pos] = i;                         // always true: the keys are those counted above
+    for (int base = 0; base < B; base += U * SAM_ORDER_THREADS) {
+        int key[U];
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const int i = base + u * SAM_ORDER_THREADS + (int)threadIdx.x;
+            key[u] = i < B ? keys[i] : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            const int i = base + u * SAM_ORDER_THREADS + (int)threadIdx.x;
+            const unsigned peers = __match_any_sync(FULL, key[u]);
+            const int leader = __ffs(peers) - 1;
+            int pos = 0;
+            if (key[u] >= 0 && lane == leader) pos = atomicAdd(&hist[key[u]], __popc(peers));
+            pos = __shfl_sync(FULL, pos, leader) + __popc(peers & lt);
+            if (key[u] >= 0 && pos < B) order[pos] = i;      // always true: the keys are those counted above
+        }
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
@@ -1506,6 +1564,7 @@ int split_kernel_setup(int device) {
     if (device < 0 || device >= 64) return SAM_ERR_ARG;
     if (!done[device]) {
         cudaError_t e = cudaFuncSetAttribute(sam_step_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(order_slots_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, 50);
         if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
         done[device] = true;
     }
@@ -1555,10 +1614,15 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
         int32_t* order = b->view.order + (size_t)(b->order_phase & 1) * b->view.batch;
         cudaLaunchConfig_t oc;
         memset(&oc, 0, sizeof(oc));
-        oc.gridDim = dim3(1); oc.blockDim = dim3(1024); oc.stream = stream; oc.attrs = attr; oc.numAttrs = 1;
+        oc.gridDim = dim3(1); oc.blockDim = dim3(SAM_ORDER_THREADS); oc.stream = stream; oc.attrs = attr; oc.numAttrs = 1;
         int32_t* n_big = b->view.order + 3 * (size_t)b->view.batch + 8 * (b->order_phase & 1);
-        cudaError_t oe = cudaLaunchKernelEx(&oc, order_slots_kernel, counts, (int32_t)b->view.batch, order,
-                                            b->view.order + 2 * (size_t)b->view.batch, split_big_m(b->view.batch), n_big);
+        const bool split = A.has_static && b->view.batch >= SAM_SPLIT_MIN_BATCH;
+        if (split) { int rc = split_kernel_setup(b->device); if (rc) return rc; }
+        cudaError_t oe = split
+            ? cudaLaunchKernelEx(&oc, order_slots_kernel<true>, counts, (int32_t)b->view.batch, order,
+                                 b->view.order + 2 * (size_t)b->view.batch, split_big_m(b->view.batch), n_big)
+            : cudaLaunchKernelEx(&oc, order_slots_kernel<false>, counts, (int32_t)b->view.batch, order,
+                                 b->view.order + 2 * (size_t)b->view.batch, split_big_m(b->view.batch), n_big);
         A.split_count = n_big;
         b->order_phase ^= 1;
         if (oe != cudaSuccess) { sam_set_cuda_error(oe); return SAM_ERR_CUDA; }

@@ -127,19 +127,21 @@ def test_fused_verify_and_step_matches_the_two_call_loop(P):
         P.binding.sam_step_verified(batch.handle, target, new.draft_tokens, new.draft_len, cap, L, *new.tensors())
 
 
-def _large_loop_case():
-    spec = W.scaled(W.SPECS["c5"], 150_000, 1600, 40, 60)
+def _large_loop_case(batch):
+    spec = W.scaled(W.SPECS["c5"], 150_000, batch, 40, 60)
     w = W.make(spec)
     return spec, w
 
 
-def test_two_call_loop_above_the_slot_ordering_threshold(P):
+# 1600 slots: the step kernel preceded by the slot-ordering kernel; 8300 slots: the split step
+@pytest.mark.parametrize("n_slots", [1600, 8300])
+def test_two_call_loop_above_the_slot_ordering_threshold(P, n_slots):
     """The closed loop with a batch large enough for the slot-ordering kernel (two launches per step):
     the counts each step reads were written by the kernel just before it on the stream
     (sam_accept_greedy), which is the case the ordering kernel must tolerate.  Step for step equal to
     the oracle's loop."""
     import torch
-    spec, w = _large_loop_case()
+    spec, w = _large_loop_case(n_slots)
     B, pl, L = spec.batch, spec.prompt_len, spec.draft_len
     total, stride = pl + spec.gen_len, L + 1
     S = oracle.Sam(w.corpus)
@@ -172,12 +174,13 @@ def test_two_call_loop_above_the_slot_ordering_threshold(P):
     assert np.array_equal(pos.cpu().numpy(), pos_ref) and (pos_ref == total).all()
 
 
-def test_counts_written_by_the_fused_step_feed_a_plain_step(P):
+@pytest.mark.parametrize("n_slots", [1600, 8300])
+def test_counts_written_by_the_fused_step_feed_a_plain_step(P, n_slots):
     """sam_step_verified writes counts_out; the very next call on the stream is a sam_step that takes
     that array as its counts (feeding as many tokens of the continuation again).  With 1600 slots the
     plain step sorts its slots by those counts first.  Every output equals the oracle fed the same way."""
     import torch
-    spec, w = _large_loop_case()
+    spec, w = _large_loop_case(n_slots)
     B, pl, L = spec.batch, spec.prompt_len, spec.draft_len
     total = pl + spec.gen_len
     S = oracle.Sam(w.corpus)

@@ -246,6 +246,44 @@ def test_large_batch_is_ordered_by_token_count(P):
     assert_dynamic_automata_equal(batch, ob, [0, 777, spec.batch - 1], msl)
 
 
+@pytest.mark.parametrize("l_bias,min_match,stop", [(0, 1, -1), (2, 3, 7)])
+def test_split_step_for_very_large_batches(P, l_bias, min_match, stop):
+    """From 8192 slots on a step runs as the split kernel: the static side of a slot in one block (a lane
+    or a warp of it, by token count), the dynamic side in another, the outputs written by whichever
+    finishes last.  Every output of every step equals the oracle's, slot for slot, and so do sampled
+    dynamic automata; counts include 0 and the prompt is fed in one step (hundreds of tokens per slot)."""
+    spec = W.scaled(W.SPECS["c5"], 200_000, 8300, 130, 90)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    counts = w.counts.copy()
+    counts[3, ::7] = 0                                      # some slots sit a step out (their tokens are dropped)
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, ob, _ = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, counts, L, msl, l_bias, min_match,
+                            threads=8, stop_token=stop)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, counts, L, msl, l_bias, min_match, stop_token=stop)
+    assert batch.launches_per_step() == 2
+    assert_same(got, ref, "split step")
+    assert (got["status"] == 0).all()
+    assert (got["source"] == 1).any() and (got["source"] == 2).any()
+    assert_dynamic_automata_equal(batch, ob, [0, 4097, spec.batch - 1], msl)
+
+
+def test_split_step_reports_failed_slots_like_the_oracle(P):
+    """Bad counts, bad tokens and texts that outgrow max_seq_len in a batch of 8300: the refused slots are
+    frozen with the oracle's status codes, the others are unaffected."""
+    spec = W.scaled(W.SPECS["c5"], 100_000, 8300, 24, 40)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len - 9     # the last tokens do not fit: status 1
+    counts, toks = w.counts.copy(), w.new_tokens.copy()
+    counts[1, 5] = -3; counts[2, 77] = spec.accept_max + 1          # status 4
+    toks[1, 100, 0] = spec.vocab; toks[2, 8200, 0] = -1             # status 3
+    st = P.StaticSam.build(w.corpus, spec.vocab)
+    ref, ob, _ = oracle_run(w.corpus, spec.vocab, w.prompts, toks, counts, L, msl, threads=8)
+    got, batch = gpu_run(P, st, spec.vocab, w.prompts, toks, counts, L, msl)
+    assert_same(got, ref, "split step, failures")
+    assert {1, 3, 4} <= set(np.unique(got["status"]).tolist())
+
+
 CASES = {
     # name: (spec key, corpus_len, batch, prompt_len, gen_len) — same recipes, smaller sizes
     "tiny_full": ("tiny", None, None, None, None),
