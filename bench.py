@@ -658,7 +658,24 @@ def measure_gpu(P, args, name, rank, world, local_rank, full):
     return res
 
 
-def roofline_block(res, cpu, probes):
+def device_counters(args, name):
+    """Operation counts of the timed steps from the library built with the counters (a child process:
+    the package loads one build of the library per process).  None if that fails."""
+    cmd = [sys.executable, os.path.join(ROOT, "bench_counters.py"), "--workload", name, "--warmup", str(args.warmup),
+           "--steps", str(args.steps)]
+    if name == args.workload and args.batch:
+        cmd += ["--batch", str(args.batch)]
+    if name == args.workload and args.corpus_tokens:
+        cmd += ["--corpus-tokens", str(args.corpus_tokens)]
+    try:
+        out = subprocess.run(cmd, capture_output=True, text=True, timeout=900)
+        lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+        return json.loads(lines[-1]) if out.returncode == 0 and lines else None
+    except Exception:
+        return None
+
+
+def roofline_block(res, cpu, probes, dev_counters=None):
     """The roofline object of one workload: algorithmic bytes per launch over the launch time against
     the stream-copy peak, the random-read rate and the dependent-access bound beside it."""
     name = res["base"].name
@@ -706,6 +723,18 @@ def roofline_block(res, cpu, probes):
                                       "dependent_accesses_per_sequence_step": {k: round(v, 2) for k, v in d.items()},
                                       "note": "d counts the accesses Algorithms 1 and 3 make one after the other; the kernel reads guessed states side by side where it can, so it may exceed this figure"}
             r["frac_of_concurrency_bound"] = (res["units_local"] / (res["launch_us"] * 1e-6 * res["K"])) / bound
+        if dev_counters:
+            # the same bound with the rounds of dependent reads the kernels themselves made (counters build):
+            # what the read-ahead, the runs and the prefix states leave of the algorithms' chains
+            ps = dev_counters["per_sequence_step"]
+            t_dep = probes["dependent_load_ns"]["%d_chains" % probes["chains"]] * 1e-9
+            dk = max(ps["static_rounds"], ps["dynamic_rounds"])
+            kb = res["B"] / (dk * t_dep)
+            r["latency_bound"] = {"value": kb, "unit": UNIT,
+                                  "formula": "B / (d x t_dep), d = rounds of dependent reads of the longer chain per sequence-step, counted by the kernels (library built with -DSAM_COUNTERS)",
+                                  "rounds_per_sequence_step": {"static_chain": round(ps["static_rounds"], 2), "dynamic_chain": round(ps["dynamic_rounds"], 2)},
+                                  "t_dep_ns": probes["dependent_load_ns"]["%d_chains" % probes["chains"]]}
+            r["frac_of_latency_bound"] = (res["units_local"] / (res["launch_us"] * 1e-6 * res["K"])) / kb
     return r
 
 
@@ -761,6 +790,9 @@ def main_ours(args):
     for n in names:
         results[n] = measure_gpu(P, args, n, rank, world, local_rank, full=(n == args.workload))
     gpu_part_s = time.perf_counter() - t_all
+    dev_counters = None
+    if one and rank == 0 and not args.no_probes:
+        dev_counters = device_counters(args, args.workload)      # (the oracle's automata are still being built meanwhile)
     if rank != 0:
         if world > 1:
             torch.distributed.destroy_process_group()
@@ -793,8 +825,11 @@ def main_ours(args):
         "status_all_ok": head["status_all_ok"],
         "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "graph_replay": head["graph_replay"],
         "clocks": head["clocks"],
-        "roofline": roofline_block(head, head_cpu if head_cpu and "value" in head_cpu else None, probes),
+        "roofline": roofline_block(head, head_cpu if head_cpu and "value" in head_cpu else None, probes, dev_counters),
     }
+    if dev_counters:
+        line["kernel_counters"] = {"per_sequence_step": {k: round(v, 3) for k, v in dev_counters["per_sequence_step"].items()},
+                                   "steps": dev_counters["steps"], "how": "python bench_counters.py (library built with -DSAM_COUNTERS)"}
     for k in ("tree_draft", "closed_loop"):
         if k in head:
             line[k] = head[k]

@@ -41,7 +41,8 @@ typedef enum {
     SAM_ERR_IO = -5,         /* file could not be read / written                              */
     SAM_ERR_FORMAT = -6,     /* file is not a static-automaton image, or its checksum is bad  */
     SAM_ERR_LIMIT = -7,      /* corpus or option exceeds what the layout can index            */
-    SAM_ERR_NO_DEVICE = -8   /* no usable CUDA device                                         */
+    SAM_ERR_NO_DEVICE = -8,  /* no usable CUDA device                                         */
+    SAM_ERR_UNSUPPORTED = -9 /* this build of the library lacks the feature                   */
 } sam_err_t;
 
 /* Per-sequence status written by sam_step (status_dev).  Non-zero is sticky until reset. */
@@ -361,6 +362,30 @@ int sam_probe_random_read(void* buf_dev, size_t footprint_bytes, int32_t granule
  * written into buf_dev by this call.  Synchronous.  Errors: ARG, NOMEM, CUDA. */
 int sam_probe_chase(void* buf_dev, size_t footprint_bytes, int64_t hops, int32_t chains,
                     void* stream, double* ns_per_hop);
+
+/* ---- operation counters (library built with -DSAM_COUNTERS) -------------------------------- */
+
+/* What the step kernels can count per slot: the operations the paper's algorithms are made of — the link and
+ * next moves of Transfer on the static automaton (Algorithm 1; their sum is what Appendix A.3 bounds by two per
+ * token), and of Expand on the slot's own automaton the transitions added on the suffix-link walk, the clones,
+ * the transitions a clone copies and the redirected transitions (Algorithm 3) — plus, per chain, the rounds of
+ * dependent reads it waited for (a read whose address came out of the read before it).  The regular build
+ * counts nothing and costs nothing; a second build of the same sources with -DSAM_COUNTERS does. */
+enum {
+    SAM_CNT_STATIC_ROUNDS = 0, SAM_CNT_STATIC_LINK_MOVES, SAM_CNT_STATIC_NEXT_MOVES,
+    SAM_CNT_DYNAMIC_ROUNDS, SAM_CNT_WALK_INSERTS, SAM_CNT_CLONES, SAM_CNT_COPIED_EDGES, SAM_CNT_REDIRECTS,
+    SAM_CNT_TOKENS, SAM_CNT_SEQ_STEPS,
+    SAM_N_COUNTERS = 12
+};
+
+/* 1 if this library was built with the counters, else 0. */
+int sam_counters_available(void);
+
+/* Make every later step on the current device add its counts to counters_dev, device uint64
+ * [slots, SAM_N_COUNTERS] (caller-owned, zeroed by the caller; slot i of ANY batch adds to row i, so attach one
+ * batch's array at a time); NULL with slots 0 detaches.  Synchronous with respect to the host; issue it when
+ * no step is in flight.  Errors: UNSUPPORTED in the regular build, ARG, CUDA. */
+int sam_counters_attach(uint64_t* counters_dev, int32_t slots);
 
 /* ---- diagnostics --------------------------------------------------------------------------- */
 

@@ -93,6 +93,8 @@ SIGNATURES = {
     "sam_strerror": (c_char_p, [c_int]),
     "sam_last_cuda_error": (c_int, []),
     "sam_version": (c_char_p, []),
+    "sam_counters_available": (c_int, []),
+    "sam_counters_attach": (c_int, [c_void_p, c_int32]),
 }
 
 
@@ -358,6 +360,25 @@ def sam_retrieve_noalloc(static_h, vocab, tokens, counts, L, l_bias, min_match,
                                       _dev_ptr(match_len, "match_len"), _dev_ptr(source, "source"),
                                       _dev_ptr(state, "state"), _dev_ptr(status, "status"), _stream_ptr(stream)),
            "sam_retrieve_noalloc")
+
+
+COUNTER_NAMES = ("static_rounds", "static_link_moves", "static_next_moves", "dynamic_rounds", "walk_inserts",
+                 "clones", "copied_edges", "redirects", "tokens", "seq_steps")
+N_COUNTERS = 12
+
+
+def sam_counters_available() -> bool:
+    return bool(lib().sam_counters_available())
+
+
+def sam_counters_attach(counters, slots: int = 0):
+    """counters: a zeroed torch uint64/int64 device tensor [slots, N_COUNTERS], or None to detach."""
+    if counters is None:
+        _check(lib().sam_counters_attach(None, 0), "sam_counters_attach")
+    else:
+        assert counters.is_cuda and counters.is_contiguous() and counters.element_size() == 8
+        assert counters.numel() >= slots * N_COUNTERS
+        _check(lib().sam_counters_attach(counters.data_ptr(), slots), "sam_counters_attach")
 
 
 def sam_probe_random_read(buf, granule: int, iters: int = 5, stream=None):

@@ -131,6 +131,7 @@ extern "C" const char* sam_strerror(int err) {
         case SAM_ERR_FORMAT: return "not a static-automaton image or checksum mismatch";
         case SAM_ERR_LIMIT: return "size exceeds what the layout can index";
         case SAM_ERR_NO_DEVICE: return "no usable CUDA device";
+        case SAM_ERR_UNSUPPORTED: return "this build of the library lacks the feature";
         default: return "unknown error";
     }
 }

@@ -32,9 +32,39 @@
 
 #include <cstring>
 
+// Operation counters (library built with -DSAM_COUNTERS only): per slot, what its two chains did — the
+// moves and insertions Algorithms 1 and 3 count, and the rounds of dependent reads each chain waited for.
+// They exist to be compared with the CPU oracle's counters and to put a number on the latency bound;
+// the regular build carries none of this.
+#ifdef SAM_COUNTERS
+__device__ unsigned long long* g_sam_counters = nullptr;     // [slots][SAM_N_COUNTERS]
+__device__ int g_sam_counter_slots = 0;
+#define SAM_COUNT(x, n) ((x) += (n))
+#else
+#define SAM_COUNT(x, n) ((void)0)
+#endif
+
 namespace {
 
 constexpr unsigned FULL = 0xFFFFFFFFu;
+
+// counts of one chain of one slot in one step (registers; dropped by the compiler in the regular build)
+struct ChainCounts { uint32_t rounds, a, b, c, d; };
+
+__device__ __forceinline__ void flush_counts(int slot, int lane, bool is_static, const ChainCounts& k, int m) {
+#ifdef SAM_COUNTERS
+    if (g_sam_counters && lane == 0 && slot < g_sam_counter_slots) {
+        unsigned long long* o = g_sam_counters + (size_t)slot * SAM_N_COUNTERS;
+        if (is_static) {
+            o[SAM_CNT_STATIC_ROUNDS] += k.rounds; o[SAM_CNT_STATIC_LINK_MOVES] += k.a; o[SAM_CNT_STATIC_NEXT_MOVES] += k.b;
+        } else {
+            o[SAM_CNT_DYNAMIC_ROUNDS] += k.rounds; o[SAM_CNT_WALK_INSERTS] += k.a; o[SAM_CNT_CLONES] += k.b;
+            o[SAM_CNT_COPIED_EDGES] += k.c; o[SAM_CNT_REDIRECTS] += k.d;
+            o[SAM_CNT_TOKENS] += (unsigned)m; o[SAM_CNT_SEQ_STEPS] += m > 0 ? 1u : 0u;
+        }
+    }
+#endif
+}
 constexpr int MAX_DRAFT_REGS = 4;     // 4 x 32 lanes = 128 draft tokens
 
 struct StepArgs {
@@ -108,12 +138,12 @@ __device__ __forceinline__ int cut_at_stop(int32_t d[MAX_DRAFT_REGS], int dl, in
 // if have_ent, pent is this lane's entry of the home bucket of (s, t), read earlier.
 __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t& s, uint32_t& sf, int32_t& l,
                                                 uint32_t t, uint32_t root_e, int lane, int& err,
-                                                bool have_rec, uint4 pa, uint4 pb, bool have_ent, uint4 pent) {
+                                                bool have_rec, uint4 pa, uint4 pb, bool have_ent, uint4 pent, ChainCounts& kc) {
     int guard = l + 2;                       // at most l link moves
     bool len_from_rec = false;
     for (;;) {
         if (s == 0) {                        // at the root the match length is 0
-            if (root_e != SAM_NONE) { s = root_e & SAM_IDMASK; sf = root_e >> 31; l = 1; }
+            if (root_e != SAM_NONE) { s = root_e & SAM_IDMASK; sf = root_e >> 31; l = 1; SAM_COUNT(kc.b, 1); }
             else l = 0;
             return;
         }
@@ -122,14 +152,14 @@ __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t
         if (sf) ent = have_ent ? pent : __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
         have_ent = false;
         uint4 a = pa, b = pb;
-        if (!have_rec) { a = __ldg(S.rec + 2 * (size_t)s); b = __ldg(S.rec + 2 * (size_t)s + 1); }
+        if (!have_rec) { a = __ldg(S.rec + 2 * (size_t)s); b = __ldg(S.rec + 2 * (size_t)s + 1); SAM_COUNT(kc.rounds, 1); }
         have_rec = false;
         if (len_from_rec) { l = (int32_t)a.x; len_from_rec = false; }
         uint32_t tgt = SAM_NONE;
         if (a.w >= 1 && b.x == t) tgt = b.y;
         else if (a.w >= 2 && b.z == t) tgt = b.w;
         else if (a.w > 2) {
-            if (!sf) ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+            if (!sf) { ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7)); SAM_COUNT(kc.rounds, 1); }
             for (int probe = 1;; probe++) {
                 unsigned hit = __ballot_sync(FULL, ent.x == s && ent.y == t);
                 if (hit) { tgt = __shfl_sync(FULL, ent.z, __ffs(hit) - 1); break; }
@@ -137,9 +167,11 @@ __device__ __forceinline__ void static_transfer(const SamStaticView& S, uint32_t
                 if (empty || probe >= S.hash_max_probe) break;
                 home = (home + 1) & S.hash_mask;
                 ent = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + (lane & 7));
+                SAM_COUNT(kc.rounds, 1);
             }
         }
-        if (tgt != SAM_NONE) { s = tgt & SAM_IDMASK; sf = tgt >> 31; l += 1; return; }
+        if (tgt != SAM_NONE) { s = tgt & SAM_IDMASK; sf = tgt >> 31; l += 1; SAM_COUNT(kc.b, 1); return; }
+        SAM_COUNT(kc.a, 1);
         s = a.y & SAM_IDMASK; sf = a.y >> 31;            // s <- link(s), l <- len(link(s))
         if (s == 0) l = 0; else len_from_rec = true;
         if (--guard < 0) { err = SAM_SEQ_WALK_LIMIT; return; }
@@ -161,6 +193,7 @@ struct Dyn {
     // (root_precompute): pr_state 0 = not known (or stale), 1 = present, 2 = absent.
     uint32_t pr_state, pr_tgt, pr_slot, pr_bucket;
     int cur;                     // lane that holds the answer for the token being processed
+    mutable ChainCounts kc;      // rounds, walk-inserts, clones, copied transitions, redirects
 };
 
 struct Pre {                     // records read ahead for the clone branch of Expand, kept in shared memory
@@ -226,7 +259,7 @@ __device__ __forceinline__ Look lookup_state(const Dyn& D, uint32_t p, uint32_t 
                                              bool have_rec = false, uint4 pa = make_uint4(0, 0, 0, 0),
                                              uint4 pb = make_uint4(0, 0, 0, 0)) {
     uint4 a = pa, b = pb;
-    if (!have_rec) { const uint4* rp = rec_ptr(D, p); a = rp[0]; b = rp[1]; }
+    if (!have_rec) { const uint4* rp = rec_ptr(D, p); a = rp[0]; b = rp[1]; SAM_COUNT(D.kc.rounds, 1); }
     Look r;
     r.len = a.x; r.link = a.y; r.deg = a.w; r.b0 = b.x; r.b1 = b.y; r.b2 = b.z; r.b3 = b.w;
     r.found = false; r.tgt = 0; r.idx = 0;
@@ -238,6 +271,7 @@ __device__ __forceinline__ Look lookup_state(const Dyn& D, uint32_t p, uint32_t 
     // 128 entries per round trip: the four reads of a lane are independent and go out together
     const uint2* blk = blk_ptr(D, b.x);
     for (uint32_t base = 0; base < a.w; base += 128) {
+        SAM_COUNT(D.kc.rounds, 1);
         uint2 e[4];
 #pragma unroll
         for (int u = 0; u < 4; u++) {
@@ -337,6 +371,7 @@ __device__ __forceinline__ RootLook root_lookup(Dyn& D, uint32_t t) {
     const uint32_t cap_mask = (D.root_bmask + 1) * SAM_ROOT_BUCKET - 1;
     const uint32_t base = (sam_hash1(t) & D.root_bmask) * SAM_ROOT_BUCKET;
     for (uint32_t off = 0; off <= cap_mask; off += 32) {
+        SAM_COUNT(D.kc.rounds, 1);
         uint2 e = D.root[(base + off + D.lane) & cap_mask];
         unsigned hit = __ballot_sync(FULL, e.x == t);
         if (hit) {
@@ -373,7 +408,7 @@ __device__ __forceinline__ void redirect_walk(Dyn& D, uint32_t pp, uint32_t t, u
         if (pp == 0) {
             RootLook r2 = root_lookup(D, t);
             if (D.err) return;
-            if (r2.found && (r2.tgt & SAM_IDMASK) == q) root_retarget(D, r2.slot, cl);
+            if (r2.found && (r2.tgt & SAM_IDMASK) == q) { root_retarget(D, r2.slot, cl); SAM_COUNT(D.kc.d, 1); }
             return;
         }
         Look l2k = lookup_state(D, pp, t, first, na, nb2);
@@ -385,6 +420,7 @@ __device__ __forceinline__ void redirect_walk(Dyn& D, uint32_t pp, uint32_t t, u
             if (l2k.deg <= 2) rw2[5 + 2 * l2k.idx] = cl;
             else blk_ptr(D, l2k.b0)[l2k.idx].y = cl;
         }
+        SAM_COUNT(D.kc.d, 1);
         pp = l2k.link;
         if (--guard < 0) { D.err = SAM_SEQ_WALK_LIMIT; return; }
     }
@@ -414,6 +450,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             rl[1] = make_uint4(t, c | SAM_FLAG, 0, 0);
         }
         __syncwarp();
+        SAM_COUNT(D.kc.a, 1);
         p = s2;                                        // link[last]
     } else {
         p = 0;                                         // empty automaton: last is the root
@@ -432,6 +469,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             if (rl.found) { found = true; at_root = true; qt = rl.tgt; plen = 0; root_slot = rl.slot; }
             else {
                 root_insert(D, rl.slot, t, c | (k == 1 ? SAM_FLAG : 0u));
+                SAM_COUNT(D.kc.a, 1);
             }
             break;
         }
@@ -439,6 +477,7 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
         use_rec = false;
         if (lk.found) { found = true; qt = lk.tgt; plen = lk.len; break; }
         insert_edge(D, p, lk, t, c);                   // len[p] + 1 < k: not solid
+        SAM_COUNT(D.kc.a, 1);
         if (D.err) return;
         p = lk.link;
         if (--guard < 0) { D.err = SAM_SEQ_WALK_LIMIT; return; }
@@ -468,7 +507,9 @@ __device__ __forceinline__ void dyn_extend(Dyn& D, uint32_t t, uint32_t& last, u
             } else {
                 qa = rq[0]; qb = rq[1];
                 if (ahead) { na = rn[0]; nb2 = rn[1]; }
+                SAM_COUNT(D.kc.rounds, 1);
             }
+            SAM_COUNT(D.kc.b, 1); SAM_COUNT(D.kc.c, qa.w); SAM_COUNT(D.kc.d, 1);   // the clone, its copied transitions, p's own redirect
             uint4 nb;
             if (qa.w <= 2) {
                 nb = make_uint4(qb.x, qb.y & SAM_IDMASK, qb.z, qb.w & SAM_IDMASK);   // copies are never solid
@@ -546,6 +587,7 @@ __device__ __forceinline__ int dyn_fresh_run(Dyn& D, uint32_t tk, int j, int cnt
     const unsigned run = ((r >= 32 ? 0u : (1u << r)) - 1u) << j;
     if (bucket_peers & run) D.pr_state = 0;                   // those buckets changed
     __syncwarp();
+    SAM_COUNT(D.kc.a, 2 * r - (last == 0 ? 1 : 0));            // per token: the previous state's transition (none from the root) and the root's
     D.n_states = c0 + r; D.root_deg += r;
     last = c0 + r - 1; ntok += r;
     return r;
@@ -593,6 +635,7 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
     const uint4* ru0 = rec_ptr(D, u0 ? u0 : q0);
     uint4 qa = rq0[0], qb = rq0[1], ua = make_uint4(0, 0, 0, 0), ub = ua;
     if (u0) { ua = ru0[0]; ub = ru0[1]; }
+    SAM_COUNT(D.kc.rounds, 1);
     const unsigned same = __ballot_sync(FULL, lane < rmax && (uint32_t)tx == tkr);
     // q_0 may be `last` itself (if token j does not continue the earliest occurrence), whose record is
     // only completed by the Expand of token j: what was read of it is then not used
@@ -688,6 +731,13 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
         redirect_walk(D, xc.z, xc.x, xc.y, n0 + 2 * (uint32_t)k + 1, (int)(l0 + k) + 2, xc.z != 0, xa, xb);
     }
     if (D.err) return 0;
+    SAM_COUNT(D.kc.rounds, 2);
+    SAM_COUNT(D.kc.a, r); SAM_COUNT(D.kc.b, r); SAM_COUNT(D.kc.d, r);
+    {
+        uint32_t copied = mine ? qa.w : 0u;
+        for (int o = 16; o; o >>= 1) copied += __shfl_xor_sync(FULL, copied, o);
+        SAM_COUNT(D.kc.c, copied);
+    }
 
     const int lr = r - 1;                                      // the last clone is the new match state
     pa = make_uint4(l0 + (uint32_t)r, __shfl_sync(FULL, qa.y, lr), __shfl_sync(FULL, qa.z, lr), __shfl_sync(FULL, qa.w, lr));
@@ -705,11 +755,12 @@ __device__ __forceinline__ int dyn_repeat_run(Dyn& D, uint32_t tk, int j, int cn
 // (ra, rb) its record.  DRAFT: also fetch the draft after the state's first end position into d / my_dl
 // (requested early where the address is known early).
 template <bool DRAFT>
-__device__ __forceinline__ void static_chain(const StepArgs& A, int lane, uint32_t* cb, uint32_t cw, int32_t tok_first,
+__device__ __forceinline__ void static_chain(const StepArgs& A, int b, int lane, uint32_t* cb, uint32_t cw, int32_t tok_first,
                                              const int32_t* toks, int m, uint32_t ntok0, uint4& ra, uint4& rb,
                                              uint32_t& s_out, uint32_t& sf_out, int32_t& l_out, int& err,
                                              int32_t d[MAX_DRAFT_REGS], int32_t& my_dl) {
     const int L = A.L;
+    ChainCounts kc = {1, 0, 0, 0, 0};                    // one round already: the control words
     uint32_t s = __shfl_sync(FULL, cw, CB_S1), sf = __shfl_sync(FULL, cw, CB_S1FLAG);
     int32_t l = (int32_t)__shfl_sync(FULL, cw, CB_L1);
     bool have = s != 0;
@@ -734,6 +785,7 @@ __device__ __forceinline__ void static_chain(const StepArgs& A, int lane, uint32
         if (DRAFT) gather_draft<1>(A.S.corpus, e2, dl2, L, lane, d);
         const unsigned agree = __ballot_sync(FULL, lane < m && cx == tok_first);
         j0 = (~agree) ? __ffs(~agree) - 1 : 32;
+        SAM_COUNT(kc.rounds, 1); SAM_COUNT(kc.b, j0);
         if (j0 > 0) {
             const uint32_t ref = __shfl_sync(FULL, px, j0 - 1);
             s = ref & SAM_IDMASK; sf = ref >> 31; l += j0; have = false;
@@ -750,6 +802,7 @@ __device__ __forceinline__ void static_chain(const StepArgs& A, int lane, uint32
         uint32_t tk = 0, re = SAM_NONE;
         if (i < m) { tk = (uint32_t)(base == 0 ? tok_first : toks[i]); re = __ldg(A.S.root_row + tk); }
         const int cnt = min(32, m - base);
+        SAM_COUNT(kc.rounds, 1);
         // Most tokens end a short match: the lookup misses, the link leads to the root, and the
         // root row gives the next state u = root_row[t].  The token after that is then looked up
         // in u — a lookup whose address is known now.  Lookups k = 0..7 (state root_row[t_k],
@@ -791,11 +844,13 @@ __device__ __forceinline__ void static_chain(const StepArgs& A, int lane, uint32
                 }
             }
             static_transfer(A.S, s, sf, l, __shfl_sync(FULL, tk, j), __shfl_sync(FULL, re, j), lane, err,
-                            have || pre, pa, pb, pre, pent);
+                            have || pre, pa, pb, pre, pent, kc);
             have = false;
         }
     }
     l_out = l; s_out = s; sf_out = sf;
+    if (l > 0 && !err) SAM_COUNT(kc.rounds, (m > 0 ? 1 : 0) + (DRAFT && !drafted ? 1 : 0));
+    flush_counts(b, lane, true, kc, m);
     if (l > 0 && !err && !drafted) {
         if (m > 0) {                                    // the state moved: read its record, keep a copy
             ra = __ldg(A.S.rec + 2 * (size_t)s);
@@ -844,6 +899,7 @@ __device__ __forceinline__ void dynamic_chain(const StepArgs& A, int b, int lane
     D.slab_shift = A.W.slab_shift; D.rps_shift = A.W.slab_shift - 5;
     D.seq = b; D.lane = lane; D.err = 0;
     D.pr_state = 0; D.pr_tgt = 0; D.pr_slot = 0; D.pr_bucket = SAM_NONE; D.cur = 0;
+    D.kc = ChainCounts{1, 0, 0, 0, 0};                   // one round already: the control words
     uint32_t last = __shfl_sync(FULL, cw, CB_LAST), ntok = ntok0;
     uint32_t s2 = __shfl_sync(FULL, cw, CB_S2), l2 = __shfl_sync(FULL, cw, CB_L2);
     if (D.n_states == 0) D.n_states = 1;            // the root exists implicitly (no record is read for it)
@@ -854,6 +910,7 @@ __device__ __forceinline__ void dynamic_chain(const StepArgs& A, int b, int lane
         uint32_t tk = 0;
         if (i < m) tk = (uint32_t)(base == 0 ? tok_first : toks[i]);
         root_precompute(D, tk, i < m);              // most walks end in the root table
+        SAM_COUNT(D.kc.rounds, 1);
         const unsigned bucket_peers = __match_any_sync(FULL, D.pr_bucket);
         const int cnt = min(32, m - base);
         int j = 0;
@@ -888,11 +945,13 @@ __device__ __forceinline__ void dynamic_chain(const StepArgs& A, int b, int lane
         }
         __syncwarp();
     }
+    if (l2 > 0 && !err) SAM_COUNT(D.kc.rounds, 1);       // the draft
     if (l2 > 0 && !err && m > 0) {                      // the state moved: get its record, keep a copy
-        if (!have) { const uint4* rs = rec_ptr(D, s2); ra = rs[0]; rb = rs[1]; }
+        if (!have) { const uint4* rs = rec_ptr(D, s2); ra = rs[0]; rb = rs[1]; SAM_COUNT(D.kc.rounds, 1); }
         if (lane == 0) { reinterpret_cast<uint4*>(cb + CB_REC2)[0] = ra; reinterpret_cast<uint4*>(cb + CB_REC2)[1] = rb; }
     }
     s2_out = s2; l2_out = l2; ntok_out = ntok;
+    if (!err) flush_counts(b, lane, false, D.kc, m);
 }
 
 // Called by one thread of a block after the block's outputs are written (and made known to that
@@ -1018,7 +1077,7 @@ __global__ void __launch_bounds__(64) sam_step_kernel(const __grid_constant__ St
         // ---------------- static automaton: Transfer per token ----------------
         if (A.has_static) {
             uint32_t s, sf; int32_t l;
-            static_chain<true>(A, lane, cb, cw, tok_first, toks, m, ntok0, ra, rb, s, sf, l, err, d, my_dl);
+            static_chain<true>(A, b, lane, cb, cw, tok_first, toks, m, ntok0, ra, rb, s, sf, l, err, d, my_dl);
             my_l = l; my_s = (int32_t)s;
         }
     } else {
@@ -1266,7 +1325,9 @@ __device__ __forceinline__ void static_lanes(const StepArgs& A, int w, int lane)
     bool need_len = false;
     int j = 0, err = 0;
     int guard = l + 2 * m + 4;                           // at most l + m link moves in all (Appendix A.3)
+    [[maybe_unused]] ChainCounts kc = {2, 0, 0, 0, 0};   // two rounds already: the slot's index, its control words
     while (__any_sync(FULL, active)) {
+        if (active) SAM_COUNT(kc.rounds, 1);
         // One round of reads for every lane, none of them under a branch (lanes that took different branches
         // would otherwise wait for their reads one group after the other): a lane that does not need a line
         // reads one that every such lane shares (record 0, bucket 0, its own first token).
@@ -1286,7 +1347,7 @@ __device__ __forceinline__ void static_lanes(const StepArgs& A, int w, int lane)
             have = false;
             bool advance = false;
             if (at_root) {                                // at the root the match length is 0
-                if (re != SAM_NONE) { s = re & SAM_IDMASK; sf = re >> 31; l = 1; } else l = 0;
+                if (re != SAM_NONE) { s = re & SAM_IDMASK; sf = re >> 31; l = 1; SAM_COUNT(kc.b, 1); } else l = 0;
                 advance = true;
             } else {
                 if (need_len) { l = (int32_t)a.x; need_len = false; }
@@ -1312,11 +1373,12 @@ __device__ __forceinline__ void static_lanes(const StepArgs& A, int w, int lane)
                         for (int e = 0; e < SAM_HASH_BUCKET; e++) ent[e] = __ldg(S.hash + (size_t)home * SAM_HASH_BUCKET + e);
                     }
                 }
-                if (tgt != SAM_NONE) { s = tgt & SAM_IDMASK; sf = tgt >> 31; l += 1; advance = true; }
+                if (tgt != SAM_NONE) { s = tgt & SAM_IDMASK; sf = tgt >> 31; l += 1; advance = true; SAM_COUNT(kc.b, 1); }
                 else {                                    // s <- link(s), l <- len(link(s))
+                    SAM_COUNT(kc.a, 1);
                     s = a.y & SAM_IDMASK; sf = a.y >> 31;
                     if (s == 0) {                         // the root either has the token or not: known already
-                        if (re != SAM_NONE) { s = re & SAM_IDMASK; sf = re >> 31; l = 1; } else l = 0;
+                        if (re != SAM_NONE) { s = re & SAM_IDMASK; sf = re >> 31; l = 1; SAM_COUNT(kc.b, 1); } else l = 0;
                         advance = true;
                     } else need_len = true;
                     if (--guard < 0) { err = SAM_SEQ_WALK_LIMIT; active = false; }
@@ -1340,6 +1402,13 @@ __device__ __forceinline__ void static_lanes(const StepArgs& A, int w, int lane)
         cb[CB_S1] = s; cb[CB_L1] = (uint32_t)l; cb[CB_S1FLAG] = sf; cb[CB_NTOK_S] = ntok_s + (uint32_t)m;
     }
     if (live && err) cb[CB_ERR_S] = (uint32_t)err;
+#ifdef SAM_COUNTERS
+    if (g_sam_counters && run && b < g_sam_counter_slots) {
+        unsigned long long* o = g_sam_counters + (size_t)b * SAM_N_COUNTERS;
+        o[SAM_CNT_STATIC_ROUNDS] += kc.rounds + (l > 0 && m > 0 ? 1u : 0u);
+        o[SAM_CNT_STATIC_LINK_MOVES] += kc.a; o[SAM_CNT_STATIC_NEXT_MOVES] += kc.b;
+    }
+#endif
     bool second = false;
     if (live) {
         if (arrive_look(cb) & 1u) { atomicAdd(cb + CB_ARRIVE, 1u); second = true; }
@@ -1427,7 +1496,7 @@ __device__ __forceinline__ void static_slot(const StepArgs& A, int b, int lane) 
         uint32_t s, sf; int32_t l, dl = 0;
         int32_t d[MAX_DRAFT_REGS];
         int err = 0;
-        static_chain<false>(A, lane, cb, cw, tok_first, toks, m, ntok_s, ra, rb, s, sf, l, err, d, dl);
+        static_chain<false>(A, b, lane, cb, cw, tok_first, toks, m, ntok_s, ra, rb, s, sf, l, err, d, dl);
         if (err && lane == 0) cb[CB_ERR_S] = (uint32_t)err;
     }
     if (arrive_warp(cb, lane)) split_epilogue(A, b, lane);
@@ -1648,4 +1717,26 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { sam_set_cuda_error(e); return SAM_ERR_CUDA; }
     return SAM_OK;
+}
+
+extern "C" int sam_counters_available(void) {
+#ifdef SAM_COUNTERS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+extern "C" int sam_counters_attach(uint64_t* counters_dev, int32_t slots) {
+#ifdef SAM_COUNTERS
+    if (slots < 0 || (!counters_dev && slots > 0)) return SAM_ERR_ARG;
+    unsigned long long* p = reinterpret_cast<unsigned long long*>(counters_dev);
+    int n = counters_dev ? slots : 0;
+    SAM_CUDA(cudaMemcpyToSymbol(g_sam_counters, &p, sizeof(p)));
+    SAM_CUDA(cudaMemcpyToSymbol(g_sam_counter_slots, &n, sizeof(n)));
+    return SAM_OK;
+#else
+    (void)counters_dev; (void)slots;
+    return SAM_ERR_UNSUPPORTED;
+#endif
 }
