@@ -175,6 +175,39 @@ def test_repeated_passages_dynamic_runs(P):
             assert (got["status"] == 0).all()
 
 
+def test_periodic_passages_and_their_breaks(P):
+    """Periodic stretches (period 1 to 9, up to several hundred tokens, also re-entered later) that break off
+    with a token the passage never had: Expand then walks down the passage's suffixes a period at a time and
+    adds a transition at every state — the longest walks the workloads contain (50 to 100 suffix links).
+    Every output and the whole automaton equal the oracle's."""
+    rng = random.Random(21)
+    n = 2600
+    for vocab, kmax in [(3, 16), (12, 40), (300, 7), (5000, 64)]:
+        x, motifs = [], []
+        while len(x) < n:
+            kind = rng.random()
+            if kind < 0.5:
+                period = rng.randint(1, 9)
+                motif = rng.choice(motifs) if motifs and rng.random() < 0.4 else [rng.randrange(vocab) for _ in range(period)]
+                motifs.append(motif)
+                reps = rng.randint(2, 400 // len(motif))
+                x.extend((motif * reps)[:rng.randint(len(motif) + 1, len(motif) * reps)])
+            elif kind < 0.7 and len(x) > 20:
+                back = rng.randint(1, 9); ln = rng.randint(10, 300)     # a copy that runs into itself
+                for _ in range(ln):
+                    x.append(x[-back])
+            else:
+                x.extend(rng.randrange(vocab) for _ in range(rng.randint(1, 5)))
+        x = x[:n]
+        nt, ct = _steps_from_text(x, rng, kmax)
+        empty = np.zeros((1, 0), np.int32)
+        ref, ob, _ = oracle_run(None, vocab, empty, nt, ct, 8, n)
+        got, batch = gpu_run(P, None, vocab, empty, nt, ct, 8, n)
+        assert_same(got, ref, "vocab %d kmax %d" % (vocab, kmax))
+        assert_dynamic_automata_equal(batch, ob, [0], n)
+        assert (got["status"] == 0).all()
+
+
 def test_static_matches_in_prefix_states(P):
     """Sequences that copy long stretches of the corpus (the match soon sits in the state of a whole
     corpus prefix, so the static side advances it by comparing with the corpus), including stretches
