@@ -85,6 +85,8 @@ def parse_args(argv=None):
                     help="run the workload's recipe with this many sequences per GPU instead of its own batch (a scaling probe, not a headline)")
     ap.add_argument("--corpus-tokens", type=int, default=0,
                     help="run the workload's recipe over a corpus of this many tokens (a reduced case for profiler captures, not a headline)")
+    ap.add_argument("--prompt-len", type=int, default=0, help="run the workload's recipe with prompts of this many tokens (a reduced case)")
+    ap.add_argument("--gen-len", type=int, default=0, help="run the workload's recipe with this many generated tokens (a reduced case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probes", action="store_true")
     ap.add_argument("--no-all-workloads", action="store_true", help="measure the named workload only")
@@ -105,9 +107,23 @@ def dist_env():
             int(os.environ.get("LOCAL_RANK", "0")))
 
 
-def variant(name: str, batch: int = 0, corpus_tokens: int = 0) -> W.Spec:
+def variant(name: str, batch: int = 0, corpus_tokens: int = 0, prompt_len: int = 0, gen_len: int = 0) -> W.Spec:
     spec = W.SPECS[name]
-    return W.scaled(spec, batch=batch or None, corpus_len=corpus_tokens or None)
+    return W.scaled(spec, batch=batch or None, corpus_len=corpus_tokens or None, prompt_len=prompt_len or None,
+                    gen_len=gen_len or None)
+
+
+def named_variant(args, name: str) -> W.Spec:
+    """The recipe `name` as the command line asks for it: size options apply to the named workload only."""
+    if name != args.workload:
+        return variant(name)
+    return variant(name, args.batch, args.corpus_tokens, args.prompt_len, args.gen_len)
+
+
+def named_label(args, name: str) -> str:
+    if name != args.workload:
+        return name
+    return workload_label(name, args.batch, args.corpus_tokens, args.prompt_len, args.gen_len)
 
 
 def config_dict(base: W.Spec, label: str, world: int) -> dict:
@@ -121,12 +137,16 @@ def config_dict(base: W.Spec, label: str, world: int) -> dict:
                   "consecutive steps.  CPU arm: caches as the preceding steps leave them"}
 
 
-def workload_label(name: str, batch: int, corpus_tokens: int) -> str:
+def workload_label(name: str, batch: int, corpus_tokens: int, prompt_len: int = 0, gen_len: int = 0) -> str:
     extra = []
     if batch > 0:
         extra.append("%d sequences" % batch)
     if corpus_tokens > 0:
         extra.append("%d corpus tokens" % corpus_tokens)
+    if prompt_len > 0:
+        extra.append("prompts of %d tokens" % prompt_len)
+    if gen_len > 0:
+        extra.append("%d generated tokens" % gen_len)
     return name + (" (recipe run with %s)" % ", ".join(extra) if extra else "")
 
 
@@ -291,9 +311,8 @@ def oracle_leg(base: W.Spec, Wm: int, K: int, threads: int, single_thread_budget
     return res
 
 
-def _oracle_child(conn, name, batch, corpus_tokens, Wm, K, threads):
+def _oracle_child(conn, base, Wm, K, threads):
     try:
-        base = variant(name, batch, corpus_tokens)
         res = oracle_leg(base, Wm, K, threads, ready=lambda info: conn.send(("ready", info)),
                          wait_for_go=lambda: conn.recv())
         conn.send(("done", res))
@@ -315,16 +334,15 @@ class OracleChildren:
         self.kids = {}
         self.threads = os.cpu_count() or 1
         for name in names:
-            batch = args.batch if name == args.workload else 0
-            ctok = args.corpus_tokens if name == args.workload else 0
-            need_gb = estimate_oracle_gb(variant(name, batch, ctok))
+            base = named_variant(args, name)
+            need_gb = estimate_oracle_gb(base)
             avail = mem_available_gb()
             if avail is not None and avail < need_gb + 24:
                 self.kids[name] = ("unavailable", "host has %.0f GB available, the oracle's automaton needs about %.0f GB"
                                    % (avail, need_gb))
                 continue
             parent, child = self.ctx.Pipe()
-            p = self.ctx.Process(target=_oracle_child, args=(child, name, batch, ctok, Wm, args.steps, self.threads),
+            p = self.ctx.Process(target=_oracle_child, args=(child, base, Wm, args.steps, self.threads),
                                  daemon=True)
             p.start()
             child.close()
@@ -485,9 +503,8 @@ def measure_gpu(P, args, name, rank, world, local_rank, full):
     """One workload on this rank's GPU.  `full`: the headline treatment (graph replay, probes, clock samples)."""
     import torch
     sd = P.binding
-    is_named = name == args.workload
-    base = variant(name, args.batch if is_named else 0, args.corpus_tokens if is_named else 0)
-    label = workload_label(name, args.batch if is_named else 0, args.corpus_tokens if is_named else 0)
+    base = named_variant(args, name)
+    label = named_label(args, name)
     t0 = time.perf_counter()
     spec, corpus, seqs, counts, new_tokens = shard_workload(base, rank, world)
     inputs_s = time.perf_counter() - t0
@@ -680,10 +697,11 @@ def device_counters(args, name):
     the package loads one build of the library per process).  None if that fails."""
     cmd = [sys.executable, os.path.join(ROOT, "bench_counters.py"), "--workload", name, "--warmup", str(args.warmup),
            "--steps", str(args.steps)]
-    if name == args.workload and args.batch:
-        cmd += ["--batch", str(args.batch)]
-    if name == args.workload and args.corpus_tokens:
-        cmd += ["--corpus-tokens", str(args.corpus_tokens)]
+    if name == args.workload:
+        for flag, v in (("--batch", args.batch), ("--corpus-tokens", args.corpus_tokens), ("--prompt-len", args.prompt_len),
+                        ("--gen-len", args.gen_len)):
+            if v:
+                cmd += [flag, str(v)]
     try:
         out = subprocess.run(cmd, capture_output=True, text=True, timeout=900)
         lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
@@ -759,8 +777,8 @@ def main_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
         return 0
-    base = variant(args.workload, args.batch, args.corpus_tokens)
-    label = workload_label(args.workload, args.batch, args.corpus_tokens)
+    base = named_variant(args, args.workload)
+    label = named_label(args, args.workload)
     threads = os.cpu_count() or 1
     res = oracle_leg(base, args.warmup, args.steps, threads)
     K = res["steps"]
@@ -784,7 +802,7 @@ def main_ours(args):
     rank, world, local_rank = dist_env()
     one = world == 1
     names = [args.workload]
-    if one and not args.no_all_workloads and not args.batch and not args.corpus_tokens:
+    if one and not args.no_all_workloads and not (args.batch or args.corpus_tokens or args.prompt_len or args.gen_len):
         names += [n for n in ORDER if n != args.workload]
     kids = None
     if one and not args.no_cpu_baseline:
