@@ -2,7 +2,8 @@
 
 Seed after seed, a reduced instance of one of the five workload recipes and a random text over a tiny
 vocabulary are run through the CUDA library and through the CPU oracle; every output of every step
-and the dynamic automata, state for state, must be equal."""
+and the dynamic automata, state for state, must be equal.  Every fifth seed also runs a batch of more than
+8192 short sequences (the split step) with random l_bias / min_match / stop token and some slots sitting steps out."""
 import os
 import random
 import time
@@ -52,6 +53,23 @@ def test_randomized_parity_stress():
         assert_same(got, ref, "small text, seed %d" % seed)
         assert_dynamic_automata_equal(batch, ob, [0], n)
         batch.close()
+        if seed % 5 == 0:                                   # the split step: more than 8192 slots, short sequences
+            key = rng.choice(["c5", "c2", "c4"])
+            B = rng.choice([8200, 8333, 9000])
+            spec = W.scaled(W.SPECS[key], rng.choice([50_000, 200_000]), B, rng.choice([20, 90, 150]), rng.choice([40, 80]), seed=seed)
+            w = W.make(spec)
+            L, msl = rng.choice([4, 32, 40]), spec.prompt_len + spec.gen_len
+            counts = w.counts.copy()
+            counts[rng.randrange(counts.shape[0]), ::rng.choice([3, 11])] = 0
+            l_bias, min_match, stop = rng.choice([(0, 1, -1), (1, 2, 5), (5, 5, -1), (0, 0, 17)])
+            st = P.StaticSam.build(w.corpus, spec.vocab)
+            ref, ob, _ = oracle_run(w.corpus, spec.vocab, w.prompts, w.new_tokens, counts, L, msl, l_bias, min_match,
+                                    threads=8, stop_token=stop)
+            got, batch = gpu_run(P, st, spec.vocab, w.prompts, w.new_tokens, counts, L, msl, l_bias, min_match, stop_token=stop)
+            assert batch.launches_per_step() == 2
+            assert_same(got, ref, "split step, %s seed %d" % (key, seed))
+            assert_dynamic_automata_equal(batch, ob, [0, B // 2, B - 1], msl)
+            batch.close()
         done += 1
     print("stress: %d seeds in %.0f s" % (done, time.time() - t0))
     assert done >= 1
