@@ -27,7 +27,10 @@
 //     tokens with the corpus, its state read from the corpus' position -> state array (a prefix state's
 //     transition on the next corpus token always leads to the next prefix state);
 //   - when the batch is larger than the GPU holds at once, the slots with the most tokens are started
-//     first (order_slots_kernel).
+//     first (order_slots_kernel);
+//   - from 8192 slots on the two sides of a slot run as separate one-warp blocks (the static side of a slot
+//     with few tokens on a single lane), neither waiting for the other, and whichever finishes last writes
+//     the slot's outputs (sam_step_split_kernel, further down).
 #include "common.h"
 
 #include <cstring>
@@ -1170,18 +1173,18 @@ __device__ __forceinline__ uint32_t arrive_look(const uint32_t* cb) {
 // the count by a device-scope fence — the wait for them to be acknowledged is what that costs — and the
 // count's old value decides.
 __device__ __forceinline__ bool arrive_warp(uint32_t* cb, int lane) {
-    uint32_t seen = 0;
-    if (lane == 0) seen = arrive_look(cb);
-    seen = __shfl_sync(FULL, seen, 0);
-    if (seen & 1u) {
+    const uint32_t seen = arrive_look(cb);                 // every lane looks for itself (one request)
+    if (__all_sync(FULL, (seen & 1u) != 0)) {
         if (lane == 0) atomicAdd(cb + CB_ARRIVE, 1u);
         return true;
     }
-    __threadfence();
+    __threadfence();                                       // every lane's own stores ...
     __syncwarp();
     unsigned old = 0;
-    if (lane == 0) { old = atomicAdd(cb + CB_ARRIVE, 1u); if (old & 1u) __threadfence(); }
-    return (__shfl_sync(FULL, old, 0) & 1u) != 0;
+    if (lane == 0) { __threadfence(); old = atomicAdd(cb + CB_ARRIVE, 1u); }   // ... and, cumulatively, all of them before the count
+    old = __shfl_sync(FULL, old, 0);
+    if (old & 1u) __threadfence();                         // the other side's stores before this warp's reads of them
+    return (old & 1u) != 0;
 }
 
 // Both sides of slot b are done: choose the source (Section 3.2), read the draft, write the outputs.
