@@ -180,6 +180,29 @@ def test_host_step_large_with_pinned_and_pageable_arrays(P, B):
         b.close()
 
 
+def test_cached_static_automaton_is_built_once_then_loaded(P, tmp_path):
+    """StaticSam.cached keeps the built image under a name derived from the corpus: the first call builds and
+    saves, the second loads the same automaton, another corpus gets another file, a damaged file is rebuilt."""
+    spec = W.scaled(W.SPECS["c2"], corpus_len=90_000, batch=3, prompt_len=60, gen_len=120)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    d = str(tmp_path / "cache")
+    st1, how1 = P.StaticSam.cached(w.corpus, spec.vocab, d)
+    st2, how2 = P.StaticSam.cached(w.corpus, spec.vocab, d)
+    assert (how1, how2) == ("built", "loaded") and len(os.listdir(d)) == 1
+    r1, _ = gpu_run(P, st1, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    r2, _ = gpu_run(P, st2, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    assert_same(r2, r1)
+    other = w.corpus.copy(); other[5] = (other[5] + 1) % spec.vocab
+    _, how3 = P.StaticSam.cached(other, spec.vocab, d)
+    assert how3 == "built" and len(os.listdir(d)) == 2
+    path = os.path.join(d, sorted(os.listdir(d))[0])
+    raw = bytearray(open(path, "rb").read()); raw[len(raw) // 2] ^= 0x10
+    open(path, "wb").write(bytes(raw))
+    hows = {P.StaticSam.cached(c, spec.vocab, d)[1] for c in (w.corpus, other)}
+    assert hows == {"built", "loaded"}                      # the damaged one was rebuilt, the other loaded
+
+
 def test_image_save_load_roundtrip(P, tmp_path):
     spec = W.scaled(W.SPECS["c2"], corpus_len=120_000, batch=4, prompt_len=100, gen_len=200)
     w = W.make(spec)
