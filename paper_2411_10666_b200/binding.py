@@ -7,6 +7,7 @@ library cannot be built or loaded this module raises; there is no fallback path.
 from __future__ import annotations
 
 import ctypes
+import os
 from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32, c_int64, c_size_t, c_void_p
 
 import numpy as np
