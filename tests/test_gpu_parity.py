@@ -301,6 +301,20 @@ def test_split_step_for_very_large_batches(P, l_bias, min_match, stop):
     assert_dynamic_automata_equal(batch, ob, [0, 4097, spec.batch - 1], msl)
 
 
+def test_very_large_batch_without_a_static_automaton(P):
+    """8300 slots and no static automaton: nothing to split, the two-warp kernel runs with sorted slots;
+    the dynamic side alone drafts, as the oracle does."""
+    spec = W.scaled(W.SPECS["c4"], 1000, 8300, 100, 60)
+    w = W.make(spec)
+    L, msl = spec.draft_len, spec.prompt_len + spec.gen_len
+    ref, ob, _ = oracle_run(None, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl, threads=8)
+    got, batch = gpu_run(P, None, spec.vocab, w.prompts, w.new_tokens, w.counts, L, msl)
+    assert batch.launches_per_step() == 2
+    assert_same(got, ref, "no static automaton")
+    assert (got["source"] == 2).any() and not (got["source"] == 1).any()
+    assert_dynamic_automata_equal(batch, ob, [0, 8299], msl)
+
+
 def test_split_step_reports_failed_slots_like_the_oracle(P):
     """Bad counts, bad tokens and texts that outgrow max_seq_len in a batch of 8300: the refused slots are
     frozen with the oracle's status codes, the others are unaffected."""
