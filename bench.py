@@ -772,7 +772,7 @@ def roofline_block(res, cpu, probes, dev_counters=None):
             traffic_src = "ncu capture is of kernel sources %s, they are now %s: not reported" % (cap[2], digest)
     r = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
          "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src,
-         "kernel": "sam_step_kernel", "launch_us": res["launch_us"],
+         "kernel": "sam_step_split_kernel" if res["B"] >= 8192 else "sam_step_kernel", "launch_us": res["launch_us"],
          "algorithmic_bytes_per_sequence_step": algo_b, "algorithmic_bytes_source": algo_src,
          "sequence_steps_per_launch": per_launch}
     if ab:
