@@ -233,7 +233,9 @@ int sam_batch_pool_info(sam_batch_t* b, int64_t* total_slabs, int64_t* free_slab
 
 /* Number of kernels one sam_step launches for this batch: 1, or 2 for a batch larger than the GPU holds
  * at once (a small kernel first orders the slots so that those with the most tokens start first; the
- * step's results do not depend on it).  Returns a negative sam_err_t for a null handle. */
+ * step's results do not depend on it).  sam_step_host, being synchronous, gains nothing from the order
+ * when its kernel works on the host arrays in place, and then makes one launch whatever the batch.
+ * Returns a negative sam_err_t for a null handle. */
 int sam_batch_launches_per_step(const sam_batch_t* b);
 
 /* Forget the batch.  The workspace is the caller's and is not freed. */

@@ -1682,7 +1682,9 @@ int sam_launch_step_full(const sam_batch* b, const int32_t* new_tokens, int32_t 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     A.order = nullptr; A.split_count = nullptr;
-    if (!v_draft && b->view.batch >= SAM_ORDER_MIN_BATCH) {
+    // (A host-array step is synchronous: nothing runs before it that the ordering kernel could overlap with, so it
+    // would cost more than the order saves; such a step is always the one two-warp launch, slots in their own order.)
+    if (!v_draft && !done_flag_dev && b->view.batch >= SAM_ORDER_MIN_BATCH) {
         int32_t* order = b->view.order + (size_t)(b->order_phase & 1) * b->view.batch;
         cudaLaunchConfig_t oc;
         memset(&oc, 0, sizeof(oc));

@@ -155,9 +155,9 @@ def test_host_step_equals_device_step(P):
 @pytest.mark.parametrize("B", [600, 1700, 8300])
 def test_host_step_large_with_pinned_and_pageable_arrays(P, B):
     """Large host steps: page-locked caller arrays are read and written in place, pageable ones go
-    through the staging area (and, at this size, two DMA copies or the mapped staging area); at 1700
-    slots the slot-ordering kernel reads the counts from host memory too, at 8300 the split step writes
-    each slot's rows from whichever block finishes it last.  All equal the oracle."""
+    through the staging area (and, at this size, two DMA copies or the mapped staging area — the DMA path
+    runs the device step as it is: slot ordering at 1700 slots, the split step at 8300; the in-place paths
+    run one unordered two-warp launch whatever the batch).  All equal the oracle."""
     import torch
     spec = W.scaled(W.SPECS["c5"], corpus_len=60_000, batch=B, prompt_len=24, gen_len=40)
     w = W.make(spec)
