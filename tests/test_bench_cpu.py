@@ -87,3 +87,26 @@ def test_multi_document_recipe_joins_documents_with_the_separator():
             assert np.array_equal(d, full[:hit[0]] if len(hit) else full)     # the plain slice, cut at the separator
             cut += len(hit) > 0
     assert cut > 0
+
+
+def test_byte_model_and_workload_naming_of_the_benchmark():
+    """The benchmark's algorithmic-byte model on hand-made counters, and the `config` object, which must be the
+    same for the GPU arm and the reference arm (both build it with the one function)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    c = dict(seq_steps=10, tokens=30, static_link_moves=5, static_next_moves=25, dynamic_link_moves=7, dynamic_next_moves=20,
+             walk_inserts=60, clones=4, copied_edges=5, redirects=6, draft_tokens=200)
+    b = bench.algorithmic_bytes(c, 32)
+    assert b["static"] == 32 * 30 / 10
+    assert b["dynamic"] == (30 * 44 + 60 * 40 + 4 * 64 + 6 * 36) / 10
+    assert b["step_io"] == (10 * (64 + 4 * 32 + 28 + 4) + 4 * 30 + 4 * 200) / 10
+    assert abs(b["total"] - (b["static"] + b["dynamic"] + b["step_io"])) < 1e-9
+    d = bench.dependent_accesses(c)
+    assert d == {"static_chain": 30 / 10 + 2, "dynamic_chain": (7 + 20 + 4 + 6) / 10 + 2}
+    a = bench.parse_args(["--workload", "c4", "--batch", "77", "--impl", "reference"])
+    spec = bench.named_variant(a, "c4")
+    assert spec.batch == 77 and bench.named_variant(a, "c2").batch == W.SPECS["c2"].batch
+    cfg = bench.config_dict(spec, bench.named_label(a, "c4"), 2)
+    assert cfg["workload"] == "c4 (recipe run with 77 sequences)" and cfg["global_batch"] == 154 and cfg["batch_per_gpu"] == 77
+    assert set(cfg) >= {"workload", "batch_per_gpu", "global_batch", "prompt_len", "gen_len", "draft_len", "corpus_tokens", "vocab", "l2"}
+    assert len(bench.kernel_digest()) == 16
